@@ -1,0 +1,288 @@
+/*
+ * antdt.h -- C-ABI boundary of the BSP sparse-ranking hot path.
+ *
+ * One synchronous (BSP) iteration of data-parallel training, as the paper's problem
+ * formulation states it (Section II): every worker i of n computes a local gradient on its
+ * local batch B_i, the servers aggregate the local gradients of all workers and update the
+ * parameters, and the global batch B = sum_i B_i is fixed (Eq. 1).  Here the n workers are
+ * simulated on one GPU, the model is the sparse-feature (embedding-bag) part of a ranking
+ * model, and the calls below are the steps of that iteration:
+ *
+ *   antdt_shard_plan         host   Stateful Dynamic Data Sharding (Section V-C) + the
+ *                                   ADJUST_BS batch sizes (Section VI-A, Eq. 2-3)
+ *   antdt_embbag_fwd         device worker forward: gather + sum pooling
+ *   antdt_embbag_bwd_dedup   device worker backward: per-worker dedup of row ids and
+ *                                   segmented reduction to mean row gradients
+ *   antdt_weighted_aggregate device server: batch-size weighted aggregation (sparse + dense)
+ *   antdt_sparse_opt_update  device server: sparse Adagrad / Adam row update
+ *
+ * Conventions
+ *   - Every call returns an int32 status (ANTDT_OK = 0).  Nothing aborts, throws or traps.
+ *   - The caller owns every buffer.  Device calls allocate no device memory; scratch is a
+ *     caller-provided workspace whose size comes from the matching *_workspace_bytes call.
+ *   - "device" pointers are CUDA global memory of the current device; "host" pointers are
+ *     ordinary host memory.  `stream` is a cudaStream_t passed as void* (NULL = legacy default
+ *     stream).  Device calls are asynchronous on that stream.
+ *   - Argument errors that the host can see are returned before anything is launched.
+ *     Errors only the device can see (row id outside [0, n_rows), offsets that do not ascend,
+ *     output capacity exceeded) are written to the caller's int32 `dev_status` word (first
+ *     error wins, the word must be zeroed by the caller before a chain of calls); the
+ *     offending element is skipped, never dereferenced.  antdt_read_status fetches it.
+ *   - Counts produced on the device stay on the device as int64 so that the chain of calls
+ *     needs no host synchronisation.
+ *   - Layout: all matrices are row-major and dense ([rows, dim], stride dim).  Bags are a CSR
+ *     list: bag b holds row_ids[bag_offsets[b] .. bag_offsets[b+1]).  Bags are ordered
+ *     sample-major (sample s, field f -> bag s*bags_per_sample + f) and the samples of worker 0
+ *     come first, then worker 1, ... (worker w owns samples
+ *     [worker_sample_offsets[w], worker_sample_offsets[w+1])).
+ *   - Limits: dim % 4 == 0 (fp32 rows) or dim % 8 == 0 (bf16 rows), dim <= 1024, all row
+ *     buffers 16-byte aligned, n_rows < 2^31, nnz < 2^31, n_bags < 2^31, n_workers <= 1024.
+ */
+#ifndef ANTDT_H
+#define ANTDT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------------------- */
+enum {
+  ANTDT_OK = 0,
+  ANTDT_ERR_INVALID_ARG = 1,         /* a host-visible argument is malformed              */
+  ANTDT_ERR_ID_OUT_OF_RANGE = 2,     /* device saw a row id outside [0, n_rows)           */
+  ANTDT_ERR_WORKSPACE_TOO_SMALL = 3, /* ws_bytes below the *_workspace_bytes figure       */
+  ANTDT_ERR_CAPACITY = 4,            /* an output buffer's capacity would be exceeded     */
+  ANTDT_ERR_CUDA = 5,                /* a CUDA runtime call or launch failed              */
+  ANTDT_ERR_TIMEOUT = 6,             /* a bounded device-side wait ran out                */
+  ANTDT_ERR_EXHAUSTED = 7,           /* the shard queue is empty: the epoch is over       */
+  ANTDT_ERR_STATE = 8,               /* call not valid in the handle's current state      */
+  ANTDT_ERR_BAD_OFFSETS = 9          /* device saw bag offsets that do not ascend / fit   */
+};
+
+enum { ANTDT_F32 = 0, ANTDT_BF16 = 1 };                  /* table row element type        */
+enum { ANTDT_RULE_PROPORTIONAL = 0, ANTDT_RULE_MINMAX = 1 };
+enum { ANTDT_OPT_ADAGRAD = 0, ANTDT_OPT_ADAM = 1 };
+enum { ANTDT_SHARD_TODO = 0, ANTDT_SHARD_DOING = 1, ANTDT_SHARD_DONE = 2 };
+
+/* ===================================================================================== */
+/* Host planner: Stateful Dynamic Data Sharding + batch-size adjustment                  */
+/* ===================================================================================== */
+
+/* A contiguous run of dataset sample indices [start, start+len).  Section V-C.1: a shard
+ * (and so every piece of one) is just two integers, start offset and length. */
+typedef struct { int64_t start, len; } antdt_range;
+
+typedef struct antdt_dds antdt_dds; /* opaque; host memory owned by the library */
+
+/* Section V-C.1.  Splits n_samples samples into ceil(n_samples / (global_batch *
+ * batches_per_shard)) shards of global_batch*batches_per_shard consecutive samples (the last
+ * one shorter), all in state TODO, and queues them in index order; shuffle_seed != 0 permutes
+ * the queue with a seeded Fisher-Yates (the "shuffle between shards" of the Shard Shuffler).
+ * *out receives the handle; release it with antdt_dds_destroy.
+ * INVALID_ARG: NULL out, n_samples < 1, global_batch < 1, batches_per_shard < 1,
+ * n_workers outside [1, 1024]. */
+int32_t antdt_dds_create(antdt_dds** out, int64_t n_samples, int64_t global_batch,
+                         int32_t batches_per_shard, int32_t n_workers, uint64_t shuffle_seed);
+void antdt_dds_destroy(antdt_dds* dds);
+
+/* Batch sizes alone (stateless).  Section VI-A: first iteration B_i = B/n (speeds == NULL,
+ * remainder to the lowest worker indices); afterwards ADJUST_BS solves Eq. 3,
+ *     min z  s.t.  z >= B_i / v_i,  sum_i B_i = B,
+ * with v_i the worker throughputs.  rule PROPORTIONAL: B_i = B*v_i/sum(v) rounded by largest
+ * remainder (ties to the lower index), workers whose share is below min_batch pinned to
+ * min_batch and the rest re-shared.  rule MINMAX: the exact integer optimum of Eq. 3 with
+ * B_i >= min_batch, built one sample at a time (each unit goes to the worker with the
+ * smallest (B_i+1)/v_i, ties to the lower index).
+ * speeds: host [n_workers] or NULL; batch_sizes: host out [n_workers], sums to global_batch.
+ * INVALID_ARG: a speed that is not finite and > 0, min_batch < 0,
+ * min_batch*n_workers > global_batch, unknown rule. */
+int32_t antdt_batch_sizes(const double* speeds, int32_t n_workers, int64_t global_batch,
+                          int32_t rule, int64_t min_batch, int64_t* batch_sizes);
+
+/* One BSP step of the data service (Sections V-C.1 to V-C.3).  Computes this step's batch
+ * sizes as antdt_batch_sizes does, then serves each worker, in ascending worker index, its
+ * batch_sizes[i] samples from the shard it currently holds; a worker whose shard runs out
+ * fetches the TODO shard at the head of the queue (it becomes DOING and cannot go to anyone
+ * else) and goes on, so a worker's step is a short list of ranges.  A shard whose last sample
+ * was served is DONE when the call returns (the step's gradients count as pushed).  When the
+ * queue is empty a worker's step is short: counts[i] < batch_sizes[i].
+ *   batch_sizes   host out [K]   planned sizes, sum = global_batch
+ *   range_offsets host out [K+1] CSR offsets into ranges
+ *   ranges        host out [ranges_cap]
+ *   counts        host out [K]   samples actually served (= batch_sizes off the epoch tail)
+ * Returns EXHAUSTED (and all counts 0) when nothing is left to serve, CAPACITY (state
+ * unchanged) when ranges_cap is too small, INVALID_ARG as antdt_batch_sizes. */
+int32_t antdt_shard_plan(antdt_dds* dds, const double* speeds, int32_t rule, int64_t min_batch,
+                         int64_t* batch_sizes, int64_t* range_offsets, antdt_range* ranges,
+                         int64_t ranges_cap, int64_t* counts);
+
+/* Section V-C.3, last paragraph: the shard a lost worker (BACKUP_WORKERS drop, KILL_RESTART)
+ * was DOING goes back to TODO at the END of the queue and will be served again in full
+ * (at-least-once).  No-op if the worker holds no shard. */
+int32_t antdt_dds_requeue_worker(antdt_dds* dds, int32_t worker);
+
+/* Shard bookkeeping used by the integrity checks (Section VII-D: #DONE = ceil(N/(B*M))). */
+int64_t antdt_dds_num_shards(const antdt_dds* dds);
+int32_t antdt_dds_counts(const antdt_dds* dds, int64_t* todo, int64_t* doing, int64_t* done);
+/* state: ANTDT_SHARD_*; owner: worker holding it or -1; r: the shard's (start, len). */
+int32_t antdt_dds_shard_info(const antdt_dds* dds, int64_t shard, int32_t* state,
+                             int32_t* owner, antdt_range* r);
+/* Serialise / restore the whole service state (the "data reading state" a checkpoint holds,
+ * Section VII-D.3).  save with buf == NULL only reports the size in *used.  load creates a
+ * new handle.  CAPACITY if cap is too small, INVALID_ARG on a malformed image. */
+int32_t antdt_dds_save(const antdt_dds* dds, void* buf, size_t cap, size_t* used);
+int32_t antdt_dds_load(antdt_dds** out, const void* buf, size_t len);
+
+/* ===================================================================================== */
+/* Device path                                                                           */
+/* ===================================================================================== */
+
+/* Worker forward (Section II: the forward part of T_i^w on the local batch B_i), for the
+ * sparse part of the model: pooled[b, :] = sum over j in bag b of table[row_ids[j], :].
+ * An id repeated inside a bag counts each time; an empty bag gives zeros.  fp32 accumulation
+ * in bag order.
+ *   table       device [n_rows, dim]  fp32 or bf16 (dtype), read only
+ *   row_ids     device [nnz]          int32 row index into table
+ *   bag_offsets device [n_bags+1]     int64, ascending, bag_offsets[0] = 0, last = nnz
+ *   pooled      device out [n_bags, dim] fp32
+ *   dev_status  device int32 word (may be NULL: errors are then only skipped) */
+int32_t antdt_embbag_fwd(const void* table, int32_t dtype, int64_t n_rows, int32_t dim,
+                         const int32_t* row_ids, int64_t nnz, const int64_t* bag_offsets,
+                         int64_t n_bags, float* pooled, int32_t* dev_status, void* stream);
+
+/* Worker backward (Section II: the backpropagation part of T_i^w; each worker produces the
+ * gradient of ITS local batch, which it then pushes).  For every worker w separately:
+ * the distinct rows its samples touch, ascending (uniq_ids), and for each of them the mean
+ * gradient over the worker's b_w = worker_sample_offsets[w+1]-worker_sample_offsets[w] samples,
+ *     uniq_grads[u, :] = (1/b_w) * sum over occurrences o of that row in worker w of
+ *                         d_pooled[bag(o), :],
+ * by a stable radix sort of the occurrences by row id and a segmented sum in sorted order --
+ * no floating-point atomics, the result is bit-reproducible from call to call.
+ *   d_pooled             device [n_bags, dim] fp32, gradient w.r.t. pooled (per-sample loss)
+ *   worker_sample_offsets host  [K+1] int64 ascending, [0] = 0, [K]*bags_per_sample = n_bags
+ *   uniq_ids             device out [out_cap] int32, grouped by worker, ascending inside one
+ *   worker_uniq_offsets  device out [K+1] int64; worker w's rows are
+ *                        [worker_uniq_offsets[w], worker_uniq_offsets[w+1]); [K] = total
+ *   seg_offsets          device out [out_cap+1] int64; the occurrences of unique row u are
+ *                        sorted positions [seg_offsets[u], seg_offsets[u+1])
+ *   sorted_occ           device out [nnz] int32; bag index of each occurrence in sorted order
+ *                        (worker, row id, then original position: all three unique)
+ *   uniq_grads           device out [out_cap, dim] fp32
+ *   out_cap              capacity in rows; nnz always suffices; CAPACITY -> dev_status
+ *   ws, ws_bytes         device scratch >= antdt_embbag_bwd_dedup_workspace_bytes(...) */
+size_t antdt_embbag_bwd_dedup_workspace_bytes(int64_t nnz, int64_t n_bags, int32_t dim,
+                                              int32_t n_workers);
+int32_t antdt_embbag_bwd_dedup(const int32_t* row_ids, int64_t nnz, const int64_t* bag_offsets,
+                               int64_t n_bags, int32_t bags_per_sample, const float* d_pooled,
+                               int32_t dim, int64_t n_rows, int32_t n_workers,
+                               const int64_t* worker_sample_offsets, int32_t* uniq_ids,
+                               int64_t* worker_uniq_offsets, int64_t* seg_offsets,
+                               int32_t* sorted_occ, float* uniq_grads, int64_t out_cap,
+                               void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* Server aggregation (Section II: "the servers aggregate the local gradients from all
+ * workers"; the global batch is fixed, Eq. 1's last constraint).  Workers push MEAN gradients
+ * over unequal local batches, so the aggregate that equals the mean over the global batch is
+ *     G = sum_i (b_i / sum_j b_j) * G_i.
+ * Sparse part: agg_ids = ascending union of the workers' row lists, a worker that does not
+ * hold a row contributes nothing; summed in ascending worker order.  Dense part: the same
+ * weights over K dense vectors.  Either part may be NULL.
+ *   batch_sizes host [K] int64: the b_i actually served this step (counts), sum > 0. */
+typedef struct {
+  int32_t dim;
+  int64_t n_rows;                     /* table rows: ids are < n_rows                      */
+  const int32_t* uniq_ids;            /* device [in_cap]      \                            */
+  const int64_t* worker_uniq_offsets; /* device [K+1]          > antdt_embbag_bwd_dedup's  */
+  const float* uniq_grads;            /* device [in_cap, dim] /  outputs                   */
+  int64_t in_cap;                     /* upper bound of worker_uniq_offsets[K]             */
+  int32_t* agg_ids;                   /* device out [out_cap]                              */
+  float* agg_grads;                   /* device out [out_cap, dim]                         */
+  int64_t* n_agg;                     /* device out, one int64                             */
+  int64_t out_cap;                    /* rows; in_cap always suffices                      */
+} antdt_sparse_part;
+
+typedef struct {
+  const float* grads; /* device [K, stride], worker i's vector at grads + i*stride        */
+  int64_t n;          /* elements per vector, n % 4 == 0                                  */
+  int64_t stride;     /* >= n, stride % 4 == 0                                            */
+  float* out;         /* device out [n]                                                   */
+} antdt_dense_part;
+
+size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32_t n_workers);
+int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                 const int64_t* batch_sizes, int32_t n_workers, void* ws,
+                                 size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* Server update (Section II: the servers "update the parameters"), on the rows in ids only;
+ * every other row of table and state is left bit-identical.
+ *   Adagrad: state0 += g*g;  w -= lr * g / (sqrt(state0) + eps)
+ *   Adam:    state0 = b1*state0 + (1-b1)*g;  state1 = b2*state1 + (1-b2)*g*g;
+ *            w -= lr * (state0/(1-b1^step)) / (sqrt(state1/(1-b2^step)) + eps)
+ * step is the global 1-based iteration.  Arithmetic is fp32; bf16 rows are widened, updated
+ * and stored back round-to-nearest-even.  ids must be distinct (aggregate's output is).
+ *   table  device [n_rows, dim] dtype, in/out      state0/state1 device [n_rows, dim] fp32
+ *   ids    device [*n_ids_dev] int32               grads  device [*n_ids_dev, dim] fp32
+ *   n_ids_dev device int64 (count stays on device); max_ids: host upper bound for it */
+int32_t antdt_sparse_opt_update(void* table, int32_t dtype, int64_t n_rows, int32_t dim,
+                                const int32_t* ids, const float* grads,
+                                const int64_t* n_ids_dev, int64_t max_ids, int32_t opt, float lr,
+                                float eps, float beta1, float beta2, int64_t step, float* state0,
+                                float* state1, int32_t* dev_status, void* stream);
+
+/* One whole step from HOST buffers: copies the step's inputs to the caller's device staging
+ * buffers, runs fwd, bwd_dedup, aggregate and update in order on `stream`, and copies the
+ * results (pooled, dense_out, n_agg, status) back; all asynchronous on `stream`, the caller
+ * synchronises.  Host buffers should be page-locked for the copies to overlap.  Every
+ * pointer of the descriptor is described beside its field. */
+typedef struct {
+  /* model state, device resident */
+  void* table; int32_t dtype; int64_t n_rows; int32_t dim;
+  float* state0; float* state1;
+  int32_t opt; float lr, eps, beta1, beta2; int64_t step;
+  /* this step's batch: host inputs */
+  const int32_t* h_row_ids; int64_t nnz;
+  const int64_t* h_bag_offsets; int64_t n_bags; int32_t bags_per_sample;
+  const float* h_d_pooled;              /* host [n_bags, dim]                              */
+  const float* h_dense_grads;           /* host [K, dense_n] or NULL                       */
+  int64_t dense_n;
+  int32_t n_workers;
+  const int64_t* worker_sample_offsets; /* host [K+1]                                      */
+  const int64_t* batch_sizes;           /* host [K]                                        */
+  /* device staging, caller allocated */
+  int32_t* d_row_ids; int64_t* d_bag_offsets; float* d_pooled_out; float* d_d_pooled;
+  float* d_dense_grads; float* d_dense_out;
+  int32_t* d_uniq_ids; int64_t* d_worker_uniq_offsets; int64_t* d_seg_offsets;
+  int32_t* d_sorted_occ; float* d_uniq_grads; int64_t uniq_cap;
+  int32_t* d_agg_ids; float* d_agg_grads; int64_t* d_n_agg; int64_t agg_cap;
+  void* ws; size_t ws_bytes;            /* >= max of the two workspace figures             */
+  int32_t* d_status;
+  /* host outputs */
+  float* h_pooled;                      /* host [n_bags, dim]                              */
+  float* h_dense_out;                   /* host [dense_n] or NULL                          */
+  int64_t* h_n_agg; int32_t* h_status;  /* one element each                                */
+} antdt_step_desc;
+int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream);
+
+/* ---- helpers ------------------------------------------------------------------------ */
+/* Synchronises `stream`, copies the status word to the host and returns it (or
+ * ANTDT_ERR_CUDA).  dev_status: device int32. */
+int32_t antdt_read_status(const int32_t* dev_status, void* stream);
+/* Number of kernels this library has launched since it was loaded. */
+int64_t antdt_launch_count(void);
+/* Per-kernel device timing: when enabled, every launch is bracketed by CUDA events on its
+ * stream.  antdt_profile_get synchronises the recorded events and reports, for kernel slot
+ * idx in [0, antdt_profile_kernels()), its name, launches and summed milliseconds since
+ * antdt_profile_enable(1). */
+int32_t antdt_profile_enable(int32_t on);
+int32_t antdt_profile_kernels(void);
+int32_t antdt_profile_get(int32_t idx, char* name, size_t name_cap, int64_t* launches,
+                          double* total_ms);
+const char* antdt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ANTDT_H */

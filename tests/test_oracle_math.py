@@ -1,0 +1,256 @@
+"""Pins of the CPU checker's device-step functions against definitions written another way:
+dense count-matrix algebra in numpy float64, closed forms, special cases and the invariants
+the aggregation must satisfy (weighted mean of worker means == mean over the global batch)."""
+import numpy as np
+import pytest
+
+import oracle
+from tests.util import bf16_bits_to_f64, count_matrix, f32_to_bf16_bits_trunc_exact, random_bags
+
+
+def _workers(rng, K, n_samples):
+    cuts = np.sort(rng.integers(0, n_samples + 1, size=K - 1))
+    return np.concatenate([[0], cuts, [n_samples]]).astype(np.int64)
+
+
+# ---- forward -----------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_fwd_equals_count_matrix_product(seed):
+    rng = np.random.default_rng(seed)
+    V, D, n_bags = 50, 8, 40
+    W = rng.normal(0, 0.01, size=(V, D)).astype(np.float32)
+    ids, off = random_bags(rng, n_bags, V, 6, zipf=1.3 if seed else None)
+    got = oracle.embbag_fwd(W, ids, off)
+    want = count_matrix(ids, off, V) @ W.astype(np.float64)
+    assert np.array_equal(got, want.astype(np.float32)) or np.allclose(got, want, rtol=1e-7, atol=0)
+    empty = np.flatnonzero(np.diff(off) == 0)
+    assert np.all(got[empty] == 0)
+
+
+def test_fwd_one_hot_returns_row_exactly_and_repeats_count():
+    rng = np.random.default_rng(5)
+    V, D = 30, 4
+    W = rng.normal(size=(V, D)).astype(np.float32)
+    ids = rng.integers(0, V, size=20).astype(np.int32)
+    off = np.arange(21, dtype=np.int64)
+    assert np.array_equal(oracle.embbag_fwd(W, ids, off), W[ids])
+    # one bag holding the same id three times = 3 * row
+    got = oracle.embbag_fwd(W, np.array([7, 7, 7], np.int32), np.array([0, 3], np.int64))
+    assert np.array_equal(got[0], (3.0 * W[7].astype(np.float64)).astype(np.float32))
+
+
+def test_fwd_bf16_rows_are_widened_exactly():
+    rng = np.random.default_rng(6)
+    V, D = 20, 8
+    bits = (rng.normal(size=(V, D)).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    ids, off = random_bags(rng, 15, V, 5)
+    got = oracle.embbag_fwd(bits, ids, off)
+    want = count_matrix(ids, off, V) @ bf16_bits_to_f64(bits)
+    assert np.allclose(got, want, rtol=1e-7, atol=0)
+
+
+def test_fwd_rejects_bad_inputs():
+    W = np.zeros((4, 4), np.float32)
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.embbag_fwd(W, np.array([4], np.int32), np.array([0, 1], np.int64))
+    assert e.value.code == 2
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.embbag_fwd(W, np.array([1, 1], np.int32), np.array([0, 2, 1], np.int64))
+    assert e.value.code == 9
+
+
+# ---- backward + dedup ----------------------------------------------------------------------
+def _brute_bwd(ids, off, F, dY, V, wso):
+    """Per worker: dW = A^T dY / b_w from the dense count matrix; lists from its columns."""
+    A = count_matrix(ids, off, V)
+    K = len(wso) - 1
+    uniq, grads, segs, wuo, occ_sorted = [], [], [0], [0], []
+    pos = 0
+    bag_of = np.repeat(np.arange(len(off) - 1), np.diff(off))
+    for w in range(K):
+        b0, b1 = wso[w] * F, wso[w + 1] * F
+        Aw = A[b0:b1]
+        dW = Aw.T @ dY[b0:b1].astype(np.float64)
+        cnt = Aw.sum(0)
+        rows = np.flatnonzero(cnt)
+        bw = float(wso[w + 1] - wso[w])
+        for r in rows:
+            uniq.append(r)
+            grads.append(dW[r] / bw)
+            pos += int(cnt[r])
+            segs.append(pos)
+        o0, o1 = off[b0], off[b1]
+        o = np.arange(o0, o1)
+        order = np.lexsort((o, ids[o0:o1]))       # by row id, then original position
+        occ_sorted.extend(bag_of[o0:o1][order].tolist())
+        wuo.append(len(uniq))
+    return (np.array(uniq, np.int32), np.array(grads, np.float64).reshape(len(uniq), -1),
+            np.array(segs, np.int64), np.array(wuo, np.int64), np.array(occ_sorted, np.int32))
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_bwd_dedup_equals_transposed_count_matrix(seed):
+    rng = np.random.default_rng(10 + seed)
+    V, D, F, K, S = 40, 4, 3, 4, 24
+    ids, off = random_bags(rng, S * F, V, 5, zipf=1.2 if seed % 2 else None)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    wso = _workers(rng, K, S)
+    if seed == 3:
+        wso = np.array([0, 0, 10, 10, S], np.int64)   # empty workers
+    r = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+    uniq, grads, segs, wuo, occ = _brute_bwd(ids, off, F, dY, V, wso)
+    assert np.array_equal(r["uniq_ids"], uniq)
+    assert np.array_equal(r["worker_uniq_offsets"], wuo)
+    assert np.array_equal(r["seg_offsets"], segs)
+    assert np.array_equal(r["sorted_occ"], occ)
+    assert np.allclose(r["uniq_grads"], grads, rtol=1e-6, atol=1e-9)
+
+
+def test_bwd_all_ids_distinct_is_a_scaled_copy():
+    rng = np.random.default_rng(20)
+    S, F, D, V = 10, 2, 4, 100
+    ids = rng.permutation(V)[: S * F].astype(np.int32)
+    off = np.arange(S * F + 1, dtype=np.int64)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    wso = np.array([0, 4, S], np.int64)
+    r = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+    for w, bw in ((0, 4.0), (1, 6.0)):
+        lo, hi = r["worker_uniq_offsets"][w], r["worker_uniq_offsets"][w + 1]
+        bags = np.arange(wso[w] * F, wso[w + 1] * F)
+        order = np.argsort(ids[bags])
+        assert np.array_equal(r["uniq_ids"][lo:hi], ids[bags][order])
+        want = (dY[bags][order].astype(np.float64) / bw).astype(np.float32)
+        assert np.array_equal(r["uniq_grads"][lo:hi], want)
+
+
+# ---- aggregation ---------------------------------------------------------------------------
+def test_weighted_aggregate_equals_full_batch_mean_gradient():
+    rng = np.random.default_rng(30)
+    V, D, F, K, S = 60, 4, 3, 5, 40
+    ids, off = random_bags(rng, S * F, V, 4, zipf=1.3)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    wso = np.array([0, 3, 11, 11, 30, S], np.int64)      # unequal batches, one empty worker
+    bsz = np.diff(wso)
+    r = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+    agg_ids, agg = oracle.aggregate_sparse(r["uniq_ids"], r["worker_uniq_offsets"],
+                                           r["uniq_grads"], bsz)
+    # forget the workers altogether: mean over the global batch
+    A = count_matrix(ids, off, V)
+    full = A.T @ dY.astype(np.float64) / float(S)
+    rows = np.flatnonzero(A.sum(0))
+    assert np.array_equal(agg_ids, rows.astype(np.int32))
+    assert np.allclose(agg, full[rows], rtol=2e-6, atol=1e-8)
+
+
+def test_aggregate_equal_batches_is_plain_mean_and_single_worker_is_identity():
+    rng = np.random.default_rng(31)
+    D, K = 4, 3
+    lists = [np.array([1, 4, 9], np.int32), np.array([4, 5], np.int32), np.array([0, 9], np.int32)]
+    uid = np.concatenate(lists)
+    wuo = np.array([0, 3, 5, 7], np.int64)
+    g = rng.normal(size=(7, D)).astype(np.float32)
+    ids, agg = oracle.aggregate_sparse(uid, wuo, g, [8, 8, 8])
+    assert ids.tolist() == [0, 1, 4, 5, 9]
+    g64 = g.astype(np.float64)
+    want = {0: g64[5] / 3, 1: g64[0] / 3, 4: (g64[1] + g64[3]) / 3, 5: g64[4] / 3,
+            9: (g64[2] + g64[6]) / 3}
+    for k, r in enumerate(ids):
+        assert np.allclose(agg[k], want[int(r)], rtol=1e-7, atol=0)
+    # unequal weights: 1/8, 3/8, 4/8 (exact in binary)
+    ids, agg = oracle.aggregate_sparse(uid, wuo, g, [1, 3, 4])
+    assert np.array_equal(agg[2], (0.125 * g64[1] + 0.375 * g64[3]).astype(np.float32))
+    # K = 1: identity, bit for bit
+    ids, agg = oracle.aggregate_sparse(lists[0], np.array([0, 3], np.int64), g[:3], [5])
+    assert np.array_equal(ids, lists[0]) and np.array_equal(agg, g[:3])
+
+
+def test_dense_aggregate_constants_and_mean():
+    bsz = np.array([64, 128, 128, 192], np.int64)
+    c = np.array([1.0, -2.0, 0.5, 4.0])
+    grads = np.repeat(c[:, None], 8, axis=1).astype(np.float32)
+    out = oracle.aggregate_dense(grads, bsz)
+    assert np.allclose(out, (bsz * c).sum() / bsz.sum(), rtol=1e-7)
+    rng = np.random.default_rng(32)
+    g = rng.normal(size=(4, 16)).astype(np.float32)
+    assert np.allclose(oracle.aggregate_dense(g, [5, 5, 5, 5]), g.astype(np.float64).mean(0),
+                       rtol=1e-6, atol=1e-9)
+    assert np.array_equal(oracle.aggregate_dense(g[:1], [3]), g[0])
+
+
+# ---- optimizers ----------------------------------------------------------------------------
+def test_adagrad_closed_form_constant_gradient():
+    V, D, T = 6, 4, 7
+    lr, eps = 0.01, 1e-8
+    W = np.full((V, D), 0.5, np.float32)
+    acc = np.zeros((V, D), np.float32)
+    g = np.array([[0.25, -0.5, 1.0, 2.0]], np.float32)
+    ids = np.array([3], np.int32)
+    for t in range(1, T + 1):
+        oracle.sparse_opt_update(W, ids, g, "adagrad", lr, eps, 0, 0, t, acc)
+    g64 = g[0].astype(np.float64)
+    # acc_T = T g^2 ;  W_T = W_0 - lr * sum_t g / (sqrt(t) |g| + eps)
+    assert np.allclose(acc[3], T * g64 ** 2, rtol=1e-6)
+    want = 0.5 - np.float64(np.float32(lr)) * sum(
+        g64 / (np.sqrt(t) * np.abs(g64) + np.float64(np.float32(eps))) for t in range(1, T + 1))
+    assert np.allclose(W[3], want, rtol=1e-6)
+    mask = np.ones(V, bool)
+    mask[3] = False
+    assert np.all(W[mask] == 0.5) and np.all(acc[mask] == 0)
+
+
+def test_zero_gradient_row_is_unchanged():
+    W = np.full((3, 4), 0.3, np.float32)
+    acc = np.full((3, 4), 2.0, np.float32)
+    oracle.sparse_opt_update(W, np.array([1], np.int32), np.zeros((1, 4), np.float32), "adagrad",
+                             0.01, 1e-8, 0, 0, 1, acc)
+    assert np.all(W == np.float32(0.3)) and np.all(acc == 2.0)
+
+
+def test_adam_first_step_and_constant_gradient_property():
+    V, D = 5, 4
+    lr, eps, b1, b2 = 1e-3, 1e-8, 0.9, 0.999
+    W = np.zeros((V, D), np.float32)
+    m = np.zeros((V, D), np.float32)
+    v = np.zeros((V, D), np.float32)
+    g = np.array([[0.5, -0.25, 3.0, -1e-3], [1.0, 1.0, -1.0, 2.0]], np.float32)
+    ids = np.array([0, 4], np.int32)
+    g64 = g.astype(np.float64)
+    step = -np.float64(np.float32(lr)) * g64 / (np.abs(g64) + np.float64(np.float32(eps)))
+    for t in range(1, 6):
+        oracle.sparse_opt_update(W, ids, g, "adam", lr, eps, b1, b2, t, m, v)
+        # m_hat = g and v_hat = g^2 at every t when g is constant: every step moves the same
+        assert np.allclose(W[ids], t * step, rtol=2e-6, atol=1e-10)
+    assert np.all(W[1:4] == 0) and np.all(m[1:4] == 0) and np.all(v[1:4] == 0)
+    b1d, b2d = np.float64(np.float32(b1)), np.float64(np.float32(b2))
+    assert np.allclose(m[ids], (1 - b1d ** 5) * g64, rtol=1e-6)
+    assert np.allclose(v[ids], (1 - b2d ** 5) * g64 ** 2, rtol=1e-6)
+
+
+def test_bf16_store_rounds_to_nearest_even():
+    # Adam, step 1, eps = 0, g = -1: the row moves by exactly +lr.  With lr = 2^-8 and bf16
+    # rows at 1.0 (ulp 2^-7) the result is an exact tie: 1.0 + 2^-8 -> even neighbour.
+    lr = 2.0 ** -8
+    start = np.array([[1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, 2.0]], np.float32)
+    even = np.array([[1.0, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -6, 2.0]], np.float32)
+    W = f32_to_bf16_bits_trunc_exact(start)
+    m = np.zeros((1, 4), np.float32)
+    v = np.zeros((1, 4), np.float32)
+    oracle.sparse_opt_update(W, np.array([0], np.int32), -np.ones((1, 4), np.float32), "adam", lr,
+                             0.0, 0.9, 0.999, 1, m, v)
+    assert np.array_equal(W, f32_to_bf16_bits_trunc_exact(even))
+    # a non-tie: +0.75 ulp rounds up, +0.25 ulp rounds down
+    for frac, up in ((0.75, True), (0.25, False)):
+        W = f32_to_bf16_bits_trunc_exact(np.array([[1.0] * 4], np.float32))
+        m[:] = 0
+        v[:] = 0
+        oracle.sparse_opt_update(W, np.array([0], np.int32), -np.ones((1, 4), np.float32), "adam",
+                                 frac * 2.0 ** -7, 0.0, 0.9, 0.999, 1, m, v)
+        want = 1.0 + 2.0 ** -7 if up else 1.0
+        assert np.all(bf16_bits_to_f64(W) == want)
+
+
+def test_update_rejects_out_of_range_id():
+    W = np.zeros((3, 4), np.float32)
+    with pytest.raises(oracle.OracleError):
+        oracle.sparse_opt_update(W, np.array([3], np.int32), np.zeros((1, 4), np.float32),
+                                 "adagrad", 0.01, 1e-8, 0, 0, 1, np.zeros((3, 4), np.float32))
