@@ -106,19 +106,24 @@ int batch_sizes(const double* v, int n, i64 B, int rule, i64 minb, i64* b) {
           --left;
         }
       }
-      // floating-point slack the other way: take back from the smallest remainders,
-      // ties to the higher index
+      // floating-point slack the other way: take back one unit each from the smallest
+      // remainders, ties to the higher index
       while (left < 0) {
-        int best = -1;
-        double bf = 2.0;
-        for (int i = 0; i < n; ++i) {
-          if (pinned[i] || b[i] <= minb) continue;
-          double fr = q[i] - std::floor(q[i]);
-          if (fr <= bf) { bf = fr; best = i; }
+        std::vector<char> used(n, 0);
+        bool progress = false;
+        for (i64 round = 0; round < n && left < 0; ++round) {
+          int best = -1;
+          double bf = 2.0;
+          for (int i = 0; i < n; ++i) {
+            if (pinned[i] || used[i]) continue;
+            double fr = q[i] - std::floor(q[i]);
+            if (fr <= bf) { bf = fr; best = i; }
+          }
+          if (best < 0) break;
+          used[best] = 1;
+          if (b[best] > minb) { b[best] -= 1; ++left; progress = true; }
         }
-        if (best < 0) return E_ARG;
-        b[best] -= 1;
-        ++left;
+        if (!progress) return E_ARG;
       }
       return OK;
     }

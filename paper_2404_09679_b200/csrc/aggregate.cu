@@ -1,0 +1,253 @@
+// Server aggregation: batch-size weighted sum of the workers' mean gradients.
+//
+// Sparse part: the workers' row lists (each ascending) are merged by one stable radix sort of
+// (row id, position in the concatenated list); equal rows then sit together in ascending
+// worker order, so one group per output row sums its <= K weighted contributions in a fixed
+// order.  Because the sorted positions of one worker ascend with the row id, the gather of the
+// workers' gradient rows is K forward-moving streams, not a random walk.
+// Dense part: a K-way streaming reduction, one 16-byte vector per thread and worker.
+#include "segsort.cuh"
+
+namespace antdt {
+namespace {
+
+constexpr int kAggThreads = 256;
+constexpr int kAggUnroll = 4;
+
+size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct AggLayout {
+  SortLayout sort;
+  size_t sort_ws, bounds, weights, wuo, keys_a, keys_b, src, vals_t, run_start, bytes;
+};
+
+AggLayout agg_layout(int64_t in_cap, int K) {
+  AggLayout L;
+  L.sort = sort_layout(1);
+  const size_t n = (size_t)(in_cap > 0 ? in_cap : 1);
+  size_t o = 0;
+  L.sort_ws = o;   o = align_up(o + L.sort.bytes);
+  L.bounds = o;    o = align_up(o + 16);
+  L.weights = o;   o = align_up(o + 4 * (size_t)K);
+  L.wuo = o;       o = align_up(o + 8 * ((size_t)K + 1));
+  L.keys_a = o;    o = align_up(o + 4 * n);
+  L.keys_b = o;    o = align_up(o + 4 * n);
+  L.src = o;       o = align_up(o + 4 * n);
+  L.vals_t = o;    o = align_up(o + 4 * n);
+  L.run_start = o; o = align_up(o + 8 * (n + 1));
+  L.bytes = o;
+  return L;
+}
+
+// bounds of the single sort segment = [0, total rows of all workers], clamped to the capacity
+__global__ void agg_prep_kernel(const int64_t* __restrict__ wuo_in, int K, int64_t in_cap,
+                                int64_t* __restrict__ bounds, int64_t* __restrict__ wuo,
+                                int32_t* status) {
+  const int tid = threadIdx.x;
+  for (int i = tid; i <= K; i += blockDim.x) {
+    int64_t v = wuo_in[i];
+    if (v < 0) v = 0;
+    if (v > in_cap) v = in_cap;
+    wuo[i] = v;
+  }
+  if (tid == 0) {
+    int64_t n = wuo_in[K];
+    if (n < 0 || n > in_cap) {
+      set_status(status, ANTDT_ERR_CAPACITY);
+      n = n < 0 ? 0 : in_cap;
+    }
+    bounds[0] = 0;
+    bounds[1] = n;
+  }
+}
+
+// One group of G lanes per output row; grid-stride because the row count lives on the device.
+template <int G, int VPL>
+__global__ void __launch_bounds__(kAggThreads)
+agg_reduce_kernel(const int64_t* __restrict__ n_agg, int64_t out_cap,
+                  const int64_t* __restrict__ run_start, const uint32_t* __restrict__ src,
+                  const int64_t* __restrict__ wuo, const float* __restrict__ weights, int K,
+                  const float* __restrict__ uniq_grads, int dim, float* __restrict__ agg_grads) {
+  extern __shared__ int64_t s_wuo[];  // [K+1], then K floats
+  float* s_w = reinterpret_cast<float*>(s_wuo + (K + 1));
+  for (int i = threadIdx.x; i <= K; i += blockDim.x) s_wuo[i] = wuo[i];
+  for (int i = threadIdx.x; i < K; i += blockDim.x) s_w[i] = weights[i];
+  __syncthreads();
+  const int lg = threadIdx.x & (G - 1);
+  const int nvec = dim / 4;
+  const int64_t n = min(*n_agg, out_cap);
+  const int64_t stride = (int64_t)gridDim.x * (kAggThreads / G);
+  for (int64_t u = (int64_t)blockIdx.x * (kAggThreads / G) + threadIdx.x / G; u < n; u += stride) {
+    const int64_t b = run_start[u], e = run_start[u + 1];
+    float4 acc[VPL];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t j = b; j < e; j += kAggUnroll) {
+      float4 v[kAggUnroll][VPL];
+      float wt[kAggUnroll];
+#pragma unroll
+      for (int t = 0; t < kAggUnroll; ++t) {
+        wt[t] = 0.f;
+        if (j + t < e) {
+          const int64_t p = (int64_t)__ldg(src + j + t);  // same address for the whole group
+          int w = interval_of(s_wuo, K + 1, p);
+          if (w > K - 1) w = K - 1;
+          wt[t] = s_w[w];
+          const float* rp = uniq_grads + (size_t)p * dim;
+#pragma unroll
+          for (int k = 0; k < VPL; ++k) {
+            const int vi = lg + k * G;
+            if (vi < nvec) v[t][k] = ldg_f4(rp + 4 * vi);
+          }
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < kAggUnroll; ++t) {
+        if (j + t >= e) break;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          if (lg + k * G >= nvec) continue;
+          acc[k].x = fmaf(wt[t], v[t][k].x, acc[k].x);
+          acc[k].y = fmaf(wt[t], v[t][k].y, acc[k].y);
+          acc[k].z = fmaf(wt[t], v[t][k].z, acc[k].z);
+          acc[k].w = fmaf(wt[t], v[t][k].w, acc[k].w);
+        }
+      }
+    }
+    float* dst = agg_grads + (size_t)u * dim;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+      const int vi = lg + k * G;
+      if (vi < nvec) reinterpret_cast<float4*>(dst)[vi] = acc[k];
+    }
+  }
+}
+
+// dense_out[e] = sum_i w_i * g_i[e], ascending i, one float4 per thread
+__global__ void __launch_bounds__(256)
+dense_wsum_kernel(const float* __restrict__ grads, int64_t n4, int64_t stride,
+                  const float* __restrict__ weights, int K, float* __restrict__ out) {
+  extern __shared__ float s_wd[];
+  for (int i = threadIdx.x; i < K; i += blockDim.x) s_wd[i] = weights[i];
+  __syncthreads();
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += step) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float* p = grads + 4 * e;
+    int i = 0;
+    for (; i + 4 <= K; i += 4) {
+      float4 v[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) v[t] = ldg_f4(p + (size_t)(i + t) * stride);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const float w = s_wd[i + t];
+        acc.x = fmaf(w, v[t].x, acc.x); acc.y = fmaf(w, v[t].y, acc.y);
+        acc.z = fmaf(w, v[t].z, acc.z); acc.w = fmaf(w, v[t].w, acc.w);
+      }
+    }
+    for (; i < K; ++i) {
+      const float4 v = ldg_f4(p + (size_t)i * stride);
+      const float w = s_wd[i];
+      acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+      acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+    }
+    reinterpret_cast<float4*>(out)[e] = acc;
+  }
+}
+
+template <int G, int VPL>
+void launch_agg_reduce(const antdt_sparse_part* sp, const AggLayout& L, char* ws, int K,
+                       cudaStream_t s) {
+  const int64_t gpb = kAggThreads / G;
+  int64_t want = (sp->out_cap + gpb - 1) / gpb;
+  const int64_t cap = (int64_t)kNumSM * 16;
+  const unsigned grid = (unsigned)(want < 1 ? 1 : (want > cap ? cap : want));
+  const size_t smem = 8 * ((size_t)K + 1) + 4 * (size_t)K;
+  ANTDT_LAUNCH("agg_reduce", (agg_reduce_kernel<G, VPL>), grid, kAggThreads, smem, s, sp->n_agg,
+               sp->out_cap, (const int64_t*)(ws + L.run_start), (const uint32_t*)(ws + L.src),
+               (const int64_t*)(ws + L.wuo), (const float*)(ws + L.weights), K, sp->uniq_grads,
+               (int)sp->dim, sp->agg_grads);
+}
+
+}  // namespace
+}  // namespace antdt
+
+extern "C" size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32_t n_workers) {
+  if (in_cap < 0 || n_workers < 1 || n_workers > antdt::kMaxSegments) return 0;
+  return antdt::agg_layout(in_cap, n_workers).bytes;
+}
+
+extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                            const int64_t* batch_sizes, int32_t n_workers, void* ws,
+                                            size_t ws_bytes, int32_t* dev_status, void* stream) {
+  using namespace antdt;
+  const int K = n_workers;
+  if (K < 1 || K > kMaxSegments || !batch_sizes || !ws || !aligned16(ws)) return ANTDT_ERR_INVALID_ARG;
+  double tot = 0.0;
+  for (int i = 0; i < K; ++i) {
+    if (batch_sizes[i] < 0) return ANTDT_ERR_INVALID_ARG;
+    tot += (double)batch_sizes[i];
+  }
+  if (!(tot > 0.0)) return ANTDT_ERR_INVALID_ARG;
+  const int64_t in_cap = sp ? sp->in_cap : 0;
+  if (sp) {
+    if (sp->dim < 4 || sp->dim > 1024 || sp->dim % 4 || sp->n_rows < 1 || sp->n_rows >= (1ll << 31) ||
+        sp->in_cap < 0 || sp->in_cap >= (1ll << 31) || sp->out_cap < 0 || !sp->worker_uniq_offsets ||
+        !sp->n_agg)
+      return ANTDT_ERR_INVALID_ARG;
+    if (sp->in_cap > 0 && (!sp->uniq_ids || !sp->uniq_grads)) return ANTDT_ERR_INVALID_ARG;
+    if (sp->out_cap > 0 && (!sp->agg_ids || !sp->agg_grads)) return ANTDT_ERR_INVALID_ARG;
+    if (!aligned16(sp->uniq_grads) || !aligned16(sp->agg_grads)) return ANTDT_ERR_INVALID_ARG;
+  }
+  if (dp) {
+    if (dp->n < 0 || dp->n % 4 || dp->stride < dp->n || dp->stride % 4) return ANTDT_ERR_INVALID_ARG;
+    if (dp->n > 0 && (!dp->grads || !dp->out || !aligned16(dp->grads) || !aligned16(dp->out)))
+      return ANTDT_ERR_INVALID_ARG;
+  }
+  const AggLayout L = agg_layout(in_cap, K);
+  if (ws_bytes < L.bytes) return ANTDT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = (cudaStream_t)stream;
+  char* w8 = static_cast<char*>(ws);
+
+  // w_i = b_i / sum_j b_j, formed in double, used in fp32
+  float hw[kMaxSegments];
+  for (int i = 0; i < K; ++i) hw[i] = (float)((double)batch_sizes[i] / tot);
+  upload_small(hw, 4 * (size_t)K, w8 + L.weights, s);
+
+  if (sp) {
+    char* sort_ws = w8 + L.sort_ws;
+    int64_t* bounds = (int64_t*)(w8 + L.bounds);
+    uint32_t* keys_a = (uint32_t*)(w8 + L.keys_a);
+    ANTDT_LAUNCH("agg_prep", agg_prep_kernel, 1, 256, 0, s, sp->worker_uniq_offsets, K, in_cap,
+                 bounds, (int64_t*)(w8 + L.wuo), dev_status);
+    segsort_setup(bounds, 1, in_cap, sort_ws, L.sort, s);
+    segsort_run(reinterpret_cast<const uint32_t*>(sp->uniq_ids), nullptr, keys_a,
+                (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b), (uint32_t*)(w8 + L.vals_t),
+                bits_for(sp->n_rows), 0, sort_ws, L.sort, dev_status, s);
+    segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
+                 sp->out_cap < in_cap ? sp->out_cap : in_cap, nullptr, nullptr, 1, sort_ws, L.sort,
+                 dev_status, s);
+    const int nvec = sp->dim / 4;
+#define AGG_CASE(G, VPL) launch_agg_reduce<G, VPL>(sp, L, w8, K, s);
+    if (nvec <= 1) { AGG_CASE(1, 1) }
+    else if (nvec <= 2) { AGG_CASE(2, 1) }
+    else if (nvec <= 4) { AGG_CASE(4, 1) }
+    else if (nvec <= 8) { AGG_CASE(8, 1) }
+    else if (nvec <= 16) { AGG_CASE(16, 1) }
+    else if (nvec <= 32) { AGG_CASE(32, 1) }
+    else if (nvec <= 64) { AGG_CASE(32, 2) }
+    else if (nvec <= 128) { AGG_CASE(32, 4) }
+    else { AGG_CASE(32, 8) }
+#undef AGG_CASE
+  }
+  if (dp && dp->n > 0) {
+    const int64_t n4 = dp->n / 4;
+    int64_t want = (n4 + 255) / 256;
+    const int64_t cap = (int64_t)kNumSM * 16;
+    const unsigned grid = (unsigned)(want > cap ? cap : want);
+    ANTDT_LAUNCH("dense_wsum", dense_wsum_kernel, grid, 256, 4 * (size_t)K, s, dp->grads, n4,
+                 dp->stride, (const float*)(w8 + L.weights), K, dp->out);
+  }
+  return cuda_ok();
+}

@@ -1,0 +1,79 @@
+// Shared device/host helpers of the CUDA translation units: launch bookkeeping, the status
+// word, 128-bit row access, group (sub-warp) shuffles.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "antdt.h"
+
+namespace antdt {
+
+// ---- launch bookkeeping (runtime.cu) --------------------------------------------------
+int prof_begin(const char* name, cudaStream_t s);
+void prof_end(int token, cudaStream_t s);
+
+// Launch `kernel` and account for it (launch counter; CUDA-event bracket when profiling is on).
+#define ANTDT_LAUNCH(name, kernel, grid, block, smem, stream, ...)        \
+  do {                                                                    \
+    int _tok = antdt::prof_begin(name, stream);                           \
+    kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);           \
+    antdt::prof_end(_tok, stream);                                        \
+  } while (0)
+
+static inline int32_t cuda_ok() {
+  return cudaGetLastError() == cudaSuccess ? ANTDT_OK : ANTDT_ERR_CUDA;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Copies a small host array (worker tables: a few KB at most) to device memory through kernel
+// parameters, 2 KB per launch, so the call neither blocks on the stream nor needs page-locked
+// memory.  bytes % 4 == 0.  Defined in runtime.cu.
+void upload_small(const void* host, size_t bytes, void* dev, cudaStream_t s);
+
+constexpr int kNumSM = 148;  // B200: 2 dies x 74 SMs; grids are sized in multiples of this
+
+// ---- device helpers -------------------------------------------------------------------
+// First error wins; a NULL status word means "skip silently".
+__device__ __forceinline__ void set_status(int32_t* st, int32_t code) {
+  if (st) atomicCAS(st, 0, code);
+}
+
+// Mask of the G-lane group this lane belongs to (G a power of two <= 32).
+template <int G>
+__device__ __forceinline__ unsigned group_mask() {
+  if (G == 32) return 0xffffffffu;
+  unsigned lane = threadIdx.x & 31u;
+  return ((1u << G) - 1u) << (lane & ~(unsigned)(G - 1));
+}
+
+__device__ __forceinline__ float4 ldg_f4(const float* p) {
+  return __ldg(reinterpret_cast<const float4*>(p));
+}
+
+// 8 bf16 (one 16-byte vector) widened to fp32; widening is exact.
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* f) {
+  f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+  f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+  f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+  f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+// Two fp32 -> packed bf16x2, round to nearest even (lo in the low half).
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// upper_bound(a[0..n), x) - 1 for ascending a with a[0] <= x: the interval that holds x.
+__device__ __forceinline__ int interval_of(const int64_t* a, int n, int64_t x) {
+  int lo = 0, hi = n;  // invariant: a[lo] <= x, (hi == n or a[hi] > x)
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (a[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+}  // namespace antdt

@@ -1,0 +1,158 @@
+// Worker forward: embedding-bag gather with sum pooling.
+//
+// One group of G lanes owns one bag; a row is read as G (x VPL) 16-byte vectors, so a warp
+// issues fully coalesced 128-bit loads over 32/G rows at once.  The bag's id list is staged
+// through the group's registers G ids at a time (one coalesced load, then shuffles), and U row
+// loads are put in flight before any is consumed.  The path is a random gather bound by HBM
+// (hot rows by L2); there is no contraction here and so no tensor-core work.
+#include "common.cuh"
+
+namespace antdt {
+namespace {
+
+constexpr int kFwdThreads = 256;
+constexpr int kFwdUnroll = 4;
+
+template <int G, int VPL, bool BF16>
+__global__ void __launch_bounds__(kFwdThreads)
+embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
+                  const int32_t* __restrict__ row_ids, int64_t nnz,
+                  const int64_t* __restrict__ bag_offsets, int64_t n_bags,
+                  float* __restrict__ pooled, int32_t* status) {
+  constexpr int EPV = BF16 ? 8 : 4;  // elements per 16-byte vector
+  const int lg = threadIdx.x & (G - 1);
+  const int64_t bag = (int64_t)blockIdx.x * (kFwdThreads / G) + (threadIdx.x / G);
+  if (bag >= n_bags) return;
+  const unsigned gmask = group_mask<G>();
+  const int nvec = dim / EPV;
+
+  int64_t begin = bag_offsets[bag], end = bag_offsets[bag + 1];
+  if (begin < 0 || end < begin || end > nnz) {  // never dereference through bad offsets
+    if (lg == 0) set_status(status, ANTDT_ERR_BAD_OFFSETS);
+    end = begin = 0;
+  }
+
+  float acc[VPL][EPV];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k)
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) acc[k][e] = 0.f;
+
+  const char* tbl = static_cast<const char*>(table);
+  const size_t row_bytes = (size_t)dim * (BF16 ? 2 : 4);
+
+  for (int64_t base = begin; base < end; base += G) {
+    const int cnt = (int)min((int64_t)G, end - base);
+    int my_id = (lg < cnt) ? __ldg(row_ids + base + lg) : -1;
+    if (lg < cnt && (my_id < 0 || (int64_t)my_id >= n_rows)) {
+      set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
+      my_id = -1;  // skipped: contributes nothing
+    }
+    for (int j = 0; j < cnt; j += kFwdUnroll) {
+      uint4 v[kFwdUnroll][VPL];
+      bool ok[kFwdUnroll];
+#pragma unroll
+      for (int u = 0; u < kFwdUnroll; ++u) {
+        // source lane stays inside the group even when j+u runs past cnt (id -1 there)
+        const int id = __shfl_sync(gmask, my_id, (j + u) & (G - 1), G);
+        ok[u] = (j + u < cnt) && id >= 0;
+        if (ok[u]) {
+          const uint4* rp = reinterpret_cast<const uint4*>(tbl + (size_t)id * row_bytes);
+#pragma unroll
+          for (int k = 0; k < VPL; ++k) {
+            const int vi = lg + k * G;
+            if (vi < nvec) v[u][k] = __ldg(rp + vi);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kFwdUnroll; ++u) {
+        if (!ok[u]) continue;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          if (lg + k * G >= nvec) continue;
+          if (BF16) {
+            float f[8];
+            bf16x8_to_f32(v[u][k], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[k][e] += f[e];
+          } else {
+            acc[k][0] += __uint_as_float(v[u][k].x);
+            acc[k][1] += __uint_as_float(v[u][k].y);
+            acc[k][2] += __uint_as_float(v[u][k].z);
+            acc[k][3] += __uint_as_float(v[u][k].w);
+          }
+        }
+      }
+    }
+  }
+
+  float* out = pooled + bag * (int64_t)dim;
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int vi = lg + k * G;
+    if (vi >= nvec) continue;
+    float4* o = reinterpret_cast<float4*>(out + (size_t)vi * EPV);
+    o[0] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+    if (BF16) o[1] = make_float4(acc[k][4], acc[k][5], acc[k][6], acc[k][7]);
+  }
+}
+
+template <int G, int VPL, bool BF16>
+void launch_fwd(const void* table, int64_t n_rows, int dim, const int32_t* row_ids, int64_t nnz,
+                const int64_t* bag_offsets, int64_t n_bags, float* pooled, int32_t* status,
+                cudaStream_t s) {
+  const int64_t gpb = kFwdThreads / G;
+  const unsigned grid = (unsigned)((n_bags + gpb - 1) / gpb);
+  ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_kernel<G, VPL, BF16>), grid, kFwdThreads, 0, s, table,
+               n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status);
+}
+
+template <bool BF16>
+int32_t dispatch_fwd(int nvec, const void* table, int64_t n_rows, int dim, const int32_t* row_ids,
+                     int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,
+                     int32_t* status, cudaStream_t s) {
+#define FWD_CASE(G, VPL)                                                                      \
+  launch_fwd<G, VPL, BF16>(table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,     \
+                           status, s);                                                        \
+  return ANTDT_OK;
+  if (nvec <= 1) { FWD_CASE(1, 1) }
+  if (nvec <= 2) { FWD_CASE(2, 1) }
+  if (nvec <= 4) { FWD_CASE(4, 1) }
+  if (nvec <= 8) { FWD_CASE(8, 1) }
+  if (nvec <= 16) { FWD_CASE(16, 1) }
+  if (nvec <= 32) { FWD_CASE(32, 1) }
+  if (nvec <= 64) { FWD_CASE(32, 2) }
+  if (nvec <= 128) { FWD_CASE(32, 4) }
+  if (nvec <= 256) { FWD_CASE(32, 8) }
+#undef FWD_CASE
+  return ANTDT_ERR_INVALID_ARG;
+}
+
+}  // namespace
+}  // namespace antdt
+
+extern "C" int32_t antdt_embbag_fwd(const void* table, int32_t dtype, int64_t n_rows, int32_t dim,
+                                    const int32_t* row_ids, int64_t nnz,
+                                    const int64_t* bag_offsets, int64_t n_bags, float* pooled,
+                                    int32_t* dev_status, void* stream) {
+  using namespace antdt;
+  if (n_bags < 0 || nnz < 0 || n_rows < 1 || n_rows >= (1ll << 31) || nnz >= (1ll << 31) ||
+      n_bags >= (1ll << 31) || dim < 1 || dim > 1024)
+    return ANTDT_ERR_INVALID_ARG;
+  if (dtype != ANTDT_F32 && dtype != ANTDT_BF16) return ANTDT_ERR_INVALID_ARG;
+  if (dim % (dtype == ANTDT_BF16 ? 8 : 4)) return ANTDT_ERR_INVALID_ARG;
+  if (n_bags == 0) return ANTDT_OK;
+  if (!table || !bag_offsets || !pooled || (nnz > 0 && !row_ids)) return ANTDT_ERR_INVALID_ARG;
+  if (!aligned16(table) || !aligned16(pooled)) return ANTDT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t rc;
+  if (dtype == ANTDT_BF16)
+    rc = dispatch_fwd<true>(dim / 8, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,
+                            dev_status, s);
+  else
+    rc = dispatch_fwd<false>(dim / 4, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags,
+                             pooled, dev_status, s);
+  if (rc != ANTDT_OK) return rc;
+  return cuda_ok();
+}

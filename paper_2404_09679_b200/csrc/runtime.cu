@@ -1,0 +1,138 @@
+// Launch accounting, per-kernel CUDA-event timing, the status word reader.
+#include <mutex>
+#include <string.h>
+#include <vector>
+
+#include "common.cuh"
+
+namespace {
+struct Slot { const char* name; int64_t launches; double ms; };
+struct Pending { int slot; cudaEvent_t a, b; };
+
+std::mutex g_mu;
+bool g_profile = false;
+int64_t g_launches = 0;
+std::vector<Slot> g_slots;
+std::vector<Pending> g_pending;
+std::vector<cudaEvent_t> g_pool;
+
+cudaEvent_t get_event() {
+  if (!g_pool.empty()) {
+    cudaEvent_t e = g_pool.back();
+    g_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+void drain_locked() {
+  for (Pending& p : g_pending) {
+    float ms = 0.f;
+    if (p.a && p.b && cudaEventSynchronize(p.b) == cudaSuccess &&
+        cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) {
+      g_slots[p.slot].ms += ms;
+    }
+    if (p.a) g_pool.push_back(p.a);
+    if (p.b) g_pool.push_back(p.b);
+  }
+  g_pending.clear();
+}
+}  // namespace
+
+namespace antdt {
+namespace {
+struct SmallBlob { uint32_t w[512]; };
+__global__ void upload_small_kernel(SmallBlob blob, int n_words, uint32_t* dst) {
+  for (int i = threadIdx.x; i < n_words; i += blockDim.x) dst[i] = blob.w[i];
+}
+}  // namespace
+
+void upload_small(const void* host, size_t bytes, void* dev, cudaStream_t s) {
+  const uint32_t* src = static_cast<const uint32_t*>(host);
+  uint32_t* dst = static_cast<uint32_t*>(dev);
+  size_t words = bytes / 4;
+  while (words > 0) {
+    SmallBlob blob;
+    const int n = (int)(words < 512 ? words : 512);
+    memcpy(blob.w, src, (size_t)n * 4);
+    ANTDT_LAUNCH("upload_small", upload_small_kernel, 1, 256, 0, s, blob, n, dst);
+    src += n;
+    dst += n;
+    words -= (size_t)n;
+  }
+}
+
+int prof_begin(const char* name, cudaStream_t s) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  ++g_launches;
+  if (!g_profile) return -1;
+  int slot = -1;
+  for (size_t i = 0; i < g_slots.size(); ++i)
+    if (g_slots[i].name == name || strcmp(g_slots[i].name, name) == 0) { slot = (int)i; break; }
+  if (slot < 0) {
+    g_slots.push_back(Slot{name, 0, 0.0});
+    slot = (int)g_slots.size() - 1;
+  }
+  g_slots[slot].launches += 1;
+  Pending p{slot, get_event(), get_event()};
+  if (p.a) cudaEventRecord(p.a, s);
+  g_pending.push_back(p);
+  return (int)g_pending.size() - 1;
+}
+
+void prof_end(int token, cudaStream_t s) {
+  if (token < 0) return;
+  std::lock_guard<std::mutex> lk(g_mu);
+  if (token < (int)g_pending.size() && g_pending[token].b) cudaEventRecord(g_pending[token].b, s);
+}
+}  // namespace antdt
+
+extern "C" {
+
+int32_t antdt_read_status(const int32_t* dev_status, void* stream) {
+  if (!dev_status) return ANTDT_ERR_INVALID_ARG;
+  int32_t h = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(&h, dev_status, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return ANTDT_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return ANTDT_ERR_CUDA;
+  return h;
+}
+
+int64_t antdt_launch_count(void) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  return g_launches;
+}
+
+int32_t antdt_profile_enable(int32_t on) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  drain_locked();
+  g_slots.clear();
+  g_profile = on != 0;
+  return ANTDT_OK;
+}
+
+int32_t antdt_profile_kernels(void) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  return (int32_t)g_slots.size();
+}
+
+int32_t antdt_profile_get(int32_t idx, char* name, size_t name_cap, int64_t* launches,
+                          double* total_ms) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  drain_locked();
+  if (idx < 0 || idx >= (int32_t)g_slots.size()) return ANTDT_ERR_INVALID_ARG;
+  if (name && name_cap) {
+    strncpy(name, g_slots[idx].name, name_cap - 1);
+    name[name_cap - 1] = 0;
+  }
+  if (launches) *launches = g_slots[idx].launches;
+  if (total_ms) *total_ms = g_slots[idx].ms;
+  return ANTDT_OK;
+}
+
+const char* antdt_version(void) { return "antdt-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,69 @@
+"""Buffer set and call sequence of one BSP step (marshalling only; all compute is in libantdt).
+
+`StepBuffers` owns the device tensors a step needs (torch = device memory only) and `run_step`
+issues the four device calls in order on the current stream.  Nothing here touches the data.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Optional, Sequence
+
+import torch
+
+from . import binding as B
+
+
+@dataclasses.dataclass
+class OptConfig:
+    opt: int
+    lr: float
+    eps: float = 1e-8
+    beta1: float = 0.9
+    beta2: float = 0.999
+
+
+class StepBuffers:
+    """Outputs, intermediates and workspace of a step, sized for at most max_nnz occurrences,
+    max_bags bags and uniq_cap (worker, row) pairs."""
+
+    def __init__(self, dim: int, n_workers: int, max_nnz: int, max_bags: int, dense_n: int = 0,
+                 uniq_cap: Optional[int] = None, agg_cap: Optional[int] = None, device="cuda"):
+        dev = torch.device(device)
+        self.dim, self.K, self.max_nnz, self.max_bags = dim, n_workers, max_nnz, max_bags
+        self.uniq_cap = max(1, uniq_cap if uniq_cap is not None else max_nnz)
+        self.agg_cap = max(1, agg_cap if agg_cap is not None else self.uniq_cap)
+        i32, i64, f32 = torch.int32, torch.int64, torch.float32
+        self.pooled = torch.empty(max(max_bags, 1), dim, dtype=f32, device=dev)
+        self.uniq_ids = torch.empty(self.uniq_cap, dtype=i32, device=dev)
+        self.worker_uniq_offsets = torch.zeros(n_workers + 1, dtype=i64, device=dev)
+        self.seg_offsets = torch.empty(self.uniq_cap + 1, dtype=i64, device=dev)
+        self.sorted_occ = torch.empty(max(max_nnz, 1), dtype=i32, device=dev)
+        self.uniq_grads = torch.empty(self.uniq_cap, dim, dtype=f32, device=dev)
+        self.agg_ids = torch.empty(self.agg_cap, dtype=i32, device=dev)
+        self.agg_grads = torch.empty(self.agg_cap, dim, dtype=f32, device=dev)
+        self.n_agg = torch.zeros(1, dtype=i64, device=dev)
+        self.status = torch.zeros(1, dtype=i32, device=dev)
+        self.dense_out = torch.empty(dense_n, dtype=f32, device=dev) if dense_n else None
+        ws_bytes = max(B.antdt_embbag_bwd_dedup_workspace_bytes(max_nnz, max_bags, dim, n_workers),
+                       B.antdt_weighted_aggregate_workspace_bytes(self.uniq_cap, n_workers))
+        self.ws = torch.empty((ws_bytes + 255) // 256 * 256, dtype=torch.uint8, device=dev)
+
+
+def run_step(buf: StepBuffers, table, state0, state1, oc: OptConfig, step: int, row_ids,
+             bag_offsets, bags_per_sample: int, d_pooled, worker_sample_offsets: Sequence[int],
+             batch_sizes: Sequence[int], dense_grads=None, stream=None):
+    """fwd -> bwd_dedup -> weighted_aggregate -> sparse_opt_update, asynchronous."""
+    n_bags = bag_offsets.numel() - 1
+    nnz = row_ids.numel()
+    B.antdt_embbag_fwd(table, row_ids, bag_offsets, buf.pooled[:n_bags], buf.status, stream)
+    B.antdt_embbag_bwd_dedup(row_ids, bag_offsets, bags_per_sample, d_pooled, table.shape[0],
+                             worker_sample_offsets, buf.uniq_ids, buf.worker_uniq_offsets,
+                             buf.seg_offsets, buf.sorted_occ[:max(nnz, 1)] if nnz else buf.sorted_occ[:0],
+                             buf.uniq_grads, buf.ws, buf.status, stream)
+    B.antdt_weighted_aggregate(batch_sizes, buf.ws, n_rows=table.shape[0], uniq_ids=buf.uniq_ids,
+                               worker_uniq_offsets=buf.worker_uniq_offsets,
+                               uniq_grads=buf.uniq_grads, agg_ids=buf.agg_ids,
+                               agg_grads=buf.agg_grads, n_agg=buf.n_agg, dense_grads=dense_grads,
+                               dense_out=buf.dense_out, dev_status=buf.status, stream=stream)
+    B.antdt_sparse_opt_update(table, buf.agg_ids, buf.agg_grads, buf.n_agg, oc.opt, oc.lr, oc.eps,
+                              oc.beta1, oc.beta2, step, state0, state1, buf.status, stream)
