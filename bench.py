@@ -1,0 +1,552 @@
+#!/usr/bin/env python
+"""Benchmark of the BSP sparse-ranking step: training samples/s per step on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+One step = planner call + embbag_fwd + embbag_bwd_dedup + weighted_aggregate + sparse_opt_update
+over one batch of seeded synthetic input.  `value` is measured with the batch resident in HBM;
+`e2e` goes through antdt_bsp_step_host with page-locked HOST buffers (copies inside the timed
+region).  The path does not shard (one GPU holds the whole table): with N > 1 every rank runs an
+independent replica and the job value is the sum of the replicas' samples over the slowest time.
+Rank 0 prints one JSON line.
+"""
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = "training samples/s per BSP step"
+UNIT = "samples/s"
+DEFAULT_CONFIG = 4          # largest single-GPU configuration (100M x 64 bf16 table, B = 131072)
+
+
+# ------------------------------------------------------------------------------------------
+# rank plumbing (torch.distributed only when launched with more than one rank)
+# ------------------------------------------------------------------------------------------
+def dist_setup(backend: str):
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group(backend=backend)
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), world
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def max_over_ranks(x: float, device="cpu") -> float:
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return x
+
+
+def sum_over_ranks(x: float, device="cpu") -> float:
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+    return x
+
+
+# ------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("uuid,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        rows = [[c.strip() for c in ln.split(",")] for ln in self.f.read().splitlines() if ln.strip()]
+        mine = [r for r in rows if len(r) >= 8 and r[0].endswith(self.uuid[-12:])] or \
+               [r for r in rows if len(r) >= 8]
+        sm, names = [], ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in mine:
+            try:
+                sm.append(float(r[1]))
+                out["sm_max_mhz"] = float(r[2])
+            except ValueError:
+                continue
+            for k, nm in enumerate(names):
+                if r[4 + k].lower().startswith("active"):
+                    reasons.add(nm)
+        if sm:
+            busy = sorted(sm)[len(sm) // 4:]          # drop idle samples around the region
+            out["sm_mhz"] = statistics.median(busy)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        return out
+
+
+# ------------------------------------------------------------------------------------------
+# workload set-up shared by both arms
+# ------------------------------------------------------------------------------------------
+def plan_all(w, n_steps):
+    from paper_2404_09679_b200 import binding as B
+    from paper_2404_09679_b200 import synth
+    dds = B.Dds(w.n_samples, w.B, w.M, w.K)
+    plans = []
+    for s in range(n_steps):
+        v = synth.speeds_for_step(w, s)
+        rc, bsz, ro, rg, cnt = dds.antdt_shard_plan(v, B.RULES[w.rule], w.min_batch)
+        assert rc == B.OK and sum(bsz) == w.B
+        plans.append(dict(speeds=v, batch_sizes=bsz, counts=cnt, ranges=rg))
+    return plans
+
+
+def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
+    """Bytes each kernel of the step has to move per launch (per step for the radix kernels'
+    sum), from the counts of the batch: the gathers at full multiplicity, every output once."""
+    D, ew = w.D, (2 if w.table_dtype == "bf16" else 4)
+    S = 2 if w.opt == "adam" else 1
+    return {
+        "embbag_fwd": 4 * nnz + 8 * (n_bags + 1) + nnz * D * ew + n_bags * D * 4,
+        "expand_bags": 8 * (n_bags + 1) + 4 * nnz,
+        "seg_reduce_tiles": 4 * nnz + nnz // 8 + nnz * D * 4 + sum_u * D * 4,
+        "agg_reduce": sum_u * (4 * D + 4) + u * (4 * D + 8),
+        "sparse_adagrad": u * (4 + 4 * D) + 2 * u * D * ew + 2 * S * u * D * 4,
+        "sparse_adam": u * (4 + 4 * D) + 2 * u * D * ew + 2 * S * u * D * 4,
+        "dense_wsum": (w.K + 1) * w.dense_n * 4,
+    }
+
+
+def step_bytes(w, nnz, n_bags, sum_u, u, passes_bwd, passes_agg):
+    b = algorithmic_bytes(w, nnz, n_bags, sum_u, u)
+    upd = b["sparse_adam"] if w.opt == "adam" else b["sparse_adagrad"]
+    sort = passes_bwd * 20 * nnz + passes_agg * 20 * sum_u + 8 * nnz + 8 * sum_u
+    return (b["embbag_fwd"] + b["expand_bags"] + b["seg_reduce_tiles"] + b["agg_reduce"] + upd +
+            (b["dense_wsum"] if w.dense_n else 0) + sort)
+
+
+# ------------------------------------------------------------------------------------------
+# CPU baseline: the checker, as it stands, on a bounded sample of the workload
+# ------------------------------------------------------------------------------------------
+class OracleSample:
+    """First `per_worker` samples of every worker of one batch, on a compact copy of the rows
+    they touch (ids renumbered in order, so every id comparison is preserved)."""
+
+    def __init__(self, w, bm, plan, table, per_worker):
+        from paper_2404_09679_b200 import synth
+        idx_parts, counts = [], []
+        ranges = list(plan["ranges"])
+        # walk the plan's ranges worker by worker
+        pos = 0
+        for i, c in enumerate(plan["counts"]):
+            take, got = min(per_worker, c), []
+            left = c
+            while left > 0:
+                s, n = ranges[pos]
+                pos += 1
+                left -= n
+                if take > 0:
+                    k = min(take, n)
+                    got.append((s, k))
+                    take -= k
+            idx_parts += got
+            counts.append(sum(n for _, n in got))
+        idx = synth.sample_indices(idx_parts, bm.device)
+        ids, off = bm.bags(idx)
+        dY = bm.d_pooled(idx)
+        rows = torch.unique(ids.to(torch.int64))          # ascending
+        self.ids = torch.searchsorted(rows, ids.to(torch.int64)).to(torch.int32).cpu().numpy()
+        self.off = off.cpu().numpy()
+        self.dY = dY.cpu().numpy()
+        t = table[rows.to(table.device)]
+        self.table = (t.view(torch.int16).cpu().numpy().view(np.uint16).copy()
+                      if t.dtype == torch.bfloat16 else t.cpu().numpy().copy())
+        self.s0 = np.zeros(self.table.shape, np.float32)
+        self.s1 = np.zeros(self.table.shape, np.float32) if w.opt == "adam" else None
+        self.counts = np.asarray(counts, np.int64)
+        self.wso = np.concatenate([[0], np.cumsum(self.counts)]).astype(np.int64)
+        dn = min(w.dense_n, 1 << 18)                    # dense part sampled in proportion
+        self.dense_frac = dn / w.dense_n if w.dense_n else 0.0
+        self.dense = None
+        if w.dense_n:
+            e = torch.arange(dn, dtype=torch.int64, device=bm.device)
+            g = [synth.normal01(synth.hash_coords(w.seed, synth.TAG_DENSE, 0, i, e)) * w.dense_std
+                 for i in range(w.K)]
+            self.dense = torch.stack(g).to(torch.float32).cpu().numpy()
+        self.w = w
+        self.n_samples = int(self.counts.sum())
+
+    def run(self, step):
+        import oracle
+        w = self.w
+        t0 = time.perf_counter()
+        oracle.embbag_fwd(self.table, self.ids, self.off)
+        b = oracle.embbag_bwd_dedup(self.ids, self.off, w.F, self.dY, self.table.shape[0], self.wso)
+        ai, ag = oracle.aggregate_sparse(b["uniq_ids"], b["worker_uniq_offsets"], b["uniq_grads"],
+                                         self.counts)
+        if self.dense is not None:
+            oracle.aggregate_dense(self.dense, self.counts)
+        oracle.sparse_opt_update(self.table, ai, ag, w.opt, w.lr, w.eps, w.beta1, w.beta2, step,
+                                 self.s0, self.s1)
+        return time.perf_counter() - t0
+
+
+# samples per worker in the bounded sample: about 15 s of checker time for the baseline leg of
+# our arm, about 5 s per step for the reference arm (which runs warmup + steps of them)
+CPU_SAMPLE_PER_WORKER = {1: 1 << 30, 2: 1 << 30, 3: 768, 4: 768, 5: 4096}
+REF_SAMPLE_PER_WORKER = {1: 1 << 30, 2: 1 << 30, 3: 256, 4: 256, 5: 1536}
+
+
+def cpu_baseline(w, cfg, bm, plan, table):
+    repeats = 5 if cfg <= 2 else 1
+    smp = OracleSample(w, bm, plan, table, CPU_SAMPLE_PER_WORKER[cfg])
+    ts = [smp.run(s + 1) for s in range(repeats)]
+    t = statistics.median(ts)
+    return {"value": smp.n_samples / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {min(CPU_SAMPLE_PER_WORKER[cfg], max(plan['counts']))} samples of each "
+                      f"of the {w.K} workers of one batch ({smp.n_samples} samples, "
+                      f"{len(smp.ids)} occurrences, touched rows only"
+                      + (f", dense vector cut to {smp.dense.shape[1]} elements" if w.dense_n else "")
+                      + f"), {repeats} step(s), {t:.2f} s per step"}, smp
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    from paper_2404_09679_b200 import binding as B
+    from paper_2404_09679_b200 import synth
+    from paper_2404_09679_b200.step import OptConfig, StepBuffers, run_step
+
+    rank, local_rank, world = dist_setup("nccl")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.lib()
+    cfg = args.config
+    w = synth.WORKLOADS[cfg]
+    if world > 1:
+        w = w.scaled(seed=w.seed + 1000 * rank)           # independent replicas
+    W, K_steps = args.warmup, args.steps
+    n_batches = min(3, W + K_steps)
+    plans = plan_all(w, max(n_batches, 1))
+    bm = synth.BatchMaker(w, dev)
+    table = bm.table()
+    state0 = torch.zeros(w.V, w.D, dtype=torch.float32, device=dev)
+    state1 = torch.zeros(w.V, w.D, dtype=torch.float32, device=dev) if w.opt == "adam" else None
+    oc = OptConfig(B.OPTS[w.opt], w.lr, w.eps, w.beta1, w.beta2)
+
+    batches = []
+    for j in range(n_batches):
+        idx = synth.sample_indices(plans[j]["ranges"], dev)
+        ids, off = bm.bags(idx)
+        batches.append(dict(ids=ids, off=off, dY=bm.d_pooled(idx), dense=bm.dense_grads(j),
+                            wso=[0] + list(np.cumsum(plans[j]["counts"])),
+                            counts=list(plans[j]["counts"])))
+        del idx
+    max_nnz = max(b["ids"].numel() for b in batches)
+    max_bags = max(b["off"].numel() - 1 for b in batches)
+
+    # CPU baseline first (rank 0, N = 1 only): it needs the initial table rows
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu, _ = cpu_baseline(w, cfg, bm, plans[0], table)
+
+    # sizing pass: count the (worker, row) pairs of every batch with capacity 0
+    ws0 = torch.empty(B.antdt_embbag_bwd_dedup_workspace_bytes(max_nnz, max_bags, w.D, w.K),
+                      dtype=torch.uint8, device=dev)
+    wuo = torch.zeros(w.K + 1, dtype=torch.int64, device=dev)
+    so = torch.zeros(1, dtype=torch.int64, device=dev)
+    occ = torch.empty(max_nnz, dtype=torch.int32, device=dev)
+    dummy = torch.empty(0, w.D, dtype=torch.float32, device=dev)
+    sum_us = []
+    for b in batches:
+        B.antdt_embbag_bwd_dedup(b["ids"], b["off"], w.F, b["dY"], w.V, b["wso"],
+                                 torch.empty(0, dtype=torch.int32, device=dev), wuo, so,
+                                 occ[: b["ids"].numel()], dummy, ws0, None)
+        sum_us.append(int(wuo[w.K].item()))
+    del ws0, occ
+    cap = int(max(sum_us) * 1.05) + 1024
+    buf = StepBuffers(w.D, w.K, max_nnz, max_bags, w.dense_n, uniq_cap=cap, agg_cap=cap, device=dev)
+
+    dds = B.Dds(w.n_samples, w.B, w.M, w.K)                # the live planner of the timed loop
+
+    def one_step(s):
+        b = batches[s % n_batches]
+        v = synth.speeds_for_step(w, s)
+        rc, bsz, _, _, cnt = dds.antdt_shard_plan(v, B.RULES[w.rule], w.min_batch)
+        if s < len(plans):
+            assert rc == B.OK and cnt == plans[s]["counts"]
+        run_step(buf, table, state0, state1, oc, s + 1, b["ids"], b["off"], w.F, b["dY"], b["wso"],
+                 b["counts"], b["dense"])
+
+    stream = torch.cuda.current_stream()
+    for s in range(W):
+        one_step(s)
+    torch.cuda.synchronize()
+    assert B.antdt_read_status(buf.status) == 0, "device status after warm-up"
+    u_seen = int(buf.n_agg.item())
+    sum_u_seen = int(buf.worker_uniq_offsets[w.K].item())
+
+    clocks = ClockSampler(local_rank)
+    barrier()
+    torch.cuda.synchronize()
+    clocks.start()
+    B.antdt_profile_enable(True)
+    launches0 = B.antdt_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(W, W + K_steps):
+        one_step(s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    ms_local = e0.elapsed_time(e1)
+    launches = B.antdt_launch_count() - launches0
+    prof = B.antdt_profile_get()
+    B.antdt_profile_enable(False)
+    clk = clocks.stop()
+    assert B.antdt_read_status(buf.status) == 0, "device status after the timed region"
+    samples_local = sum(sum(batches[s % n_batches]["counts"]) for s in range(W, W + K_steps))
+    ms = max_over_ranks(ms_local, dev)
+    samples = sum_over_ranks(float(samples_local), dev)
+
+    # ---- end to end through antdt_bsp_step_host, page-locked host buffers ---------------------
+    e2e = run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream)
+    e2e_ms = max_over_ranks(e2e["ms"], dev)
+    e2e_samples = sum_over_ranks(float(e2e["samples"]), dev)
+
+    if rank != 0:
+        return
+    # ---- roofline of the dominant kernel ---------------------------------------------------------
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except (OSError, ValueError):
+        pass
+    peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
+    nnz_avg = sum(b["ids"].numel() for b in batches) / n_batches
+    bags_avg = sum(b["off"].numel() - 1 for b in batches) / n_batches
+    alg = algorithmic_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen)
+    kern = {}
+    for name, (n, tms) in prof.items():
+        d = {"launches": n, "ms_total": round(tms, 4), "share": round(tms / max(ms_local, 1e-9), 4)}
+        if name in alg and n:
+            d["algorithmic_GBps"] = round(alg[name] / (tms / n * 1e-3) / 1e9, 1)
+        kern[name] = d
+    top = max(prof.items(), key=lambda kv: kv[1][1])[0]
+    top_n, top_ms = prof[top]
+    roof = {"kernel": top, "bound": "hbm", "unit": "GB/s", "peak": peak_gbs,
+            "peak_source": "MEASURED_PEAKS.json hbm_gbs (measured copy)" if peaks else "fallback 6650",
+            "achieved": None, "frac": None, "traffic": None,
+            "algorithmic_bytes_per_launch": alg.get(top), "avg_launch_ms": round(top_ms / top_n, 4)}
+    if top in alg:
+        roof["achieved"] = round(alg[top] / (top_ms / top_n * 1e-3) / 1e9, 1)
+        roof["frac"] = round(roof["achieved"] / peak_gbs, 4)
+    rowbits = max(1, (w.V - 1).bit_length())
+    passes = -(-rowbits // 9)
+    sb = step_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen, passes, passes)
+    line = {
+        "metric": METRIC, "value": samples / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": K_steps, "warmup": W, "ms_per_step": ms / K_steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"configs[{cfg - 1}] {w.name}: K={w.K} workers, B={w.B}, F={w.F}, "
+                               f"V={w.V} x D={w.D} {w.table_dtype}, {w.opt}",
+                   "nnz_per_step": int(nnz_avg), "bags_per_step": int(bags_avg),
+                   "uniq_worker_rows": sum_u_seen, "uniq_rows": u_seen,
+                   "l2": "no flush: per-step working set (table + state + batch) is far above the "
+                         "126 MB L2", "batches_rotated": n_batches,
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"]},
+        "e2e": {"value": e2e_samples / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "ms_per_step": e2e_ms / K_steps},
+        "gpu_launches": launches,
+        "roofline": roof,
+        "step_algorithmic_GB": round(sb / 1e9, 3),
+        "step_GBps_algorithmic": round(sb / (ms / K_steps * 1e-3) / 1e9, 1),
+        "kernels": kern,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream):
+    """K steps through antdt_bsp_step_host; every step copies its inputs from page-locked host
+    memory and its results back, and the host waits for them."""
+    def pin(t):
+        return t.cpu().pin_memory()
+
+    host = [dict(ids=pin(b["ids"]), off=pin(b["off"]), dY=pin(b["dY"]),
+                 dense=None if b["dense"] is None else pin(b["dense"])) for b in batches]
+    max_nnz = max(b["ids"].numel() for b in batches)
+    max_bags = max(b["off"].numel() - 1 for b in batches)
+    d_ids = torch.empty(max_nnz, dtype=torch.int32, device=dev)
+    d_off = torch.empty(max_bags + 1, dtype=torch.int64, device=dev)
+    d_dY = torch.empty(max_bags, w.D, dtype=torch.float32, device=dev)
+    d_dense = torch.empty(w.K, w.dense_n, dtype=torch.float32, device=dev) if w.dense_n else None
+    h_pooled = torch.empty(max_bags, w.D, dtype=torch.float32).pin_memory()
+    h_dense_out = torch.empty(w.dense_n, dtype=torch.float32).pin_memory() if w.dense_n else None
+    h_n_agg = torch.zeros(1, dtype=torch.int64).pin_memory()
+    h_status = torch.zeros(1, dtype=torch.int32).pin_memory()
+    keep = []
+
+    def desc_for(j, step):
+        b, h = batches[j], host[j]
+        wso = (C.c_int64 * (w.K + 1))(*[int(x) for x in b["wso"]])
+        bsz = (C.c_int64 * w.K)(*[int(x) for x in b["counts"]])
+        keep[:] = [wso, bsz]
+        p = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        d = B.StepDesc()
+        d.table, d.dtype, d.n_rows, d.dim = p(table), (B.BF16 if table.dtype == torch.bfloat16 else B.F32), w.V, w.D
+        d.state0, d.state1 = p(state0), p(state1)
+        d.opt, d.lr, d.eps, d.beta1, d.beta2, d.step = oc.opt, oc.lr, oc.eps, oc.beta1, oc.beta2, step
+        d.h_row_ids, d.nnz = p(h["ids"]), b["ids"].numel()
+        d.h_bag_offsets, d.n_bags, d.bags_per_sample = p(h["off"]), b["off"].numel() - 1, w.F
+        d.h_d_pooled, d.h_dense_grads, d.dense_n = p(h["dY"]), p(h["dense"]), w.dense_n
+        d.n_workers = w.K
+        d.worker_sample_offsets = C.cast(wso, C.c_void_p)
+        d.batch_sizes = C.cast(bsz, C.c_void_p)
+        d.d_row_ids, d.d_bag_offsets, d.d_pooled_out, d.d_d_pooled = p(d_ids), p(d_off), p(buf.pooled), p(d_dY)
+        d.d_dense_grads, d.d_dense_out = p(d_dense), p(buf.dense_out)
+        d.d_uniq_ids, d.d_worker_uniq_offsets = p(buf.uniq_ids), p(buf.worker_uniq_offsets)
+        d.d_seg_offsets, d.d_sorted_occ, d.d_uniq_grads = p(buf.seg_offsets), p(buf.sorted_occ), p(buf.uniq_grads)
+        d.uniq_cap = buf.uniq_cap
+        d.d_agg_ids, d.d_agg_grads, d.d_n_agg, d.agg_cap = p(buf.agg_ids), p(buf.agg_grads), p(buf.n_agg), buf.agg_cap
+        d.ws, d.ws_bytes, d.d_status = p(buf.ws), buf.ws.numel(), p(buf.status)
+        d.h_pooled, d.h_dense_out, d.h_n_agg, d.h_status = p(h_pooled), p(h_dense_out), p(h_n_agg), p(h_status)
+        return d
+
+    n_b = len(batches)
+    step0 = 10_000
+    for s in range(min(W, 3)):
+        B.antdt_bsp_step_host(desc_for(s % n_b, step0 + s), stream)
+        torch.cuda.synchronize()
+        assert int(h_status[0]) == 0
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    samples = 0
+    for s in range(K_steps):
+        j = s % n_b
+        B.antdt_bsp_step_host(desc_for(j, step0 + 3 + s), stream)
+        stream.synchronize()                              # the caller reads the step's results
+        assert int(h_status[0]) == 0 and int(h_n_agg[0]) > 0
+        samples += sum(batches[j]["counts"])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    b = batches[0]
+    h2d = (b["ids"].numel() * 4 + b["off"].numel() * 8 + b["dY"].numel() * 4 +
+           (b["dense"].numel() * 4 if b["dense"] is not None else 0))
+    d2h = (b["off"].numel() - 1) * w.D * 4 + w.dense_n * 4 + 12
+    return {"ms": e0.elapsed_time(e1), "samples": samples, "h2d": h2d, "d2h": d2h}
+
+
+# ------------------------------------------------------------------------------------------
+# reference arm: the CPU checker timed on the host cores
+# ------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2404_09679_b200 import synth
+    cfg = args.config
+    w = synth.WORKLOADS[cfg]
+    dev = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
+    plans = plan_all(w, 1)
+    bm = synth.BatchMaker(w, dev)
+
+    class _LazyTable:                     # rows of the initial table, produced on demand
+        device = dev
+        dtype = torch.float32 if w.table_dtype == "f32" else torch.bfloat16
+
+        def __getitem__(self, rows):
+            c = torch.arange(w.D, dtype=torch.int64, device=dev)
+            h = synth.hash_coords(w.seed, synth.TAG_TABLE, rows[:, None], c[None, :])
+            return (w.init_std * synth.normal01(h)).to(torch.float32).to(self.dtype)
+
+    smp = OracleSample(w, bm, plans[0], _LazyTable(), REF_SAMPLE_PER_WORKER[cfg])
+    for s in range(args.warmup):
+        smp.run(s + 1)
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        smp.run(args.warmup + s + 1)
+    dt = time.perf_counter() - t0
+    value = smp.n_samples * args.steps / dt
+    sample = (f"each step = first {min(REF_SAMPLE_PER_WORKER[cfg], max(plans[0]['counts']))} samples of "
+              f"each of the {w.K} workers of one batch ({smp.n_samples} samples, {len(smp.ids)} "
+              f"occurrences, touched rows only)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"configs[{cfg - 1}] {w.name}: K={w.K} workers, B={w.B}, F={w.F}, "
+                               f"V={w.V} x D={w.D} {w.table_dtype}, {w.opt}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
