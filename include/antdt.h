@@ -183,6 +183,37 @@ int32_t antdt_embbag_bwd_dedup(const int32_t* row_ids, int64_t nnz, const int64_
                                int32_t* sorted_occ, float* uniq_grads, int64_t out_cap,
                                void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
+/* The same backward + dedup step for callers that cannot allocate device memory.  (The paper
+ * has no counterpart: this is a packaging variant of antdt_embbag_bwd_dedup, not a step of the
+ * method.)  Some hosts of this library may not call cudaMalloc at the point where they run a
+ * step: code running inside an allocator-free real-time or serving loop, a plug-in that must live
+ * within a memory budget fixed at load time, a process whose device memory is entirely owned by
+ * another framework's pool.  For them the scratch is a fixed array of
+ * ANTDT_STATIC_SCRATCH_BYTES that lives inside the library's device image: every GPU that loads
+ * the library holds it from load to exit, whether or not this call is ever used.
+ *   - Arguments and results are those of antdt_embbag_bwd_dedup without ws / ws_bytes; inputs and
+ *     outputs are still the caller's buffers.
+ *   - Limit: antdt_embbag_bwd_dedup_workspace_bytes(nnz, n_bags, dim, n_workers) must not exceed
+ *     ANTDT_STATIC_SCRATCH_BYTES (24 MiB: roughly 1.1 million occurrences at dim 64, 1.7 million at
+ *     dim 16, with up to 64 workers).  Beyond it the call returns ANTDT_ERR_CAPACITY and launches
+ *     nothing.
+ *   - The call itself makes no cudaMalloc / cudaFree and no allocating library call.  The first
+ *     call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and find in it whatever the previous call left;
+ *     the call clears the parts that must start at zero itself.  Two calls that overlap on the
+ *     GPU (different streams, or the same stream from two threads without ordering) race on it:
+ *     serialise them. */
+#define ANTDT_STATIC_SCRATCH_BYTES (24u << 20)
+int32_t antdt_embbag_bwd_dedup_static(const int32_t* row_ids, int64_t nnz,
+                                      const int64_t* bag_offsets, int64_t n_bags,
+                                      int32_t bags_per_sample, const float* d_pooled, int32_t dim,
+                                      int64_t n_rows, int32_t n_workers,
+                                      const int64_t* worker_sample_offsets, int32_t* uniq_ids,
+                                      int64_t* worker_uniq_offsets, int64_t* seg_offsets,
+                                      int32_t* sorted_occ, float* uniq_grads, int64_t out_cap,
+                                      int32_t* dev_status, void* stream);
+
 /* Server aggregation (Section II: "the servers aggregate the local gradients from all
  * workers"; the global batch is fixed, Eq. 1's last constraint).  Workers push MEAN gradients
  * over unequal local batches, so the aggregate that equals the mean over the global batch is

@@ -29,6 +29,7 @@ EXPORTS = [
     "antdt_dds_requeue_worker", "antdt_dds_num_shards", "antdt_dds_counts", "antdt_dds_shard_info",
     "antdt_dds_save", "antdt_dds_load", "antdt_embbag_fwd",
     "antdt_embbag_bwd_dedup_workspace_bytes", "antdt_embbag_bwd_dedup",
+    "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
     "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_read_status", "antdt_launch_count",
     "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_version",
@@ -107,6 +108,9 @@ def lib() -> C.CDLL:
         L.antdt_embbag_bwd_dedup_workspace_bytes.restype = SZ
         L.antdt_embbag_bwd_dedup.argtypes = [P, I64, P, I64, I32, P, I32, I64, I32, P, P, P, P, P, P,
                                              I64, P, SZ, P, P]
+        L.antdt_embbag_bwd_dedup_static.argtypes = [P, I64, P, I64, I32, P, I32, I64, I32, P, P, P, P,
+                                                    P, P, I64, P, P]
+        L.antdt_embbag_bwd_dedup_static.restype = I32
         L.antdt_weighted_aggregate_workspace_bytes.argtypes = [I64, I32]
         L.antdt_weighted_aggregate_workspace_bytes.restype = SZ
         L.antdt_weighted_aggregate.argtypes = [P, P, P, I32, P, SZ, P, P]
@@ -262,6 +266,25 @@ def antdt_embbag_bwd_dedup(row_ids, bag_offsets, bags_per_sample: int, d_pooled,
         _dp(worker_uniq_offsets), _dp(seg_offsets), _dp(sorted_occ), _dp(uniq_grads),
         uniq_grads.shape[0], _dp(ws), ws.numel() * ws.element_size(), _dp(dev_status),
         _stream(stream)), "antdt_embbag_bwd_dedup")
+
+
+STATIC_SCRATCH_BYTES = 24 << 20
+
+
+def antdt_embbag_bwd_dedup_static(row_ids, bag_offsets, bags_per_sample: int, d_pooled, n_rows: int,
+                                  worker_sample_offsets: Sequence[int], uniq_ids, worker_uniq_offsets,
+                                  seg_offsets, sorted_occ, uniq_grads, dev_status=None, stream=None):
+    """antdt_embbag_bwd_dedup for callers that cannot allocate device memory: no workspace
+    argument, the scratch is a fixed STATIC_SCRATCH_BYTES array inside the library (shared by
+    all calls on a device, so calls must not overlap).  Raises with ERR_CAPACITY when the
+    problem needs more scratch than that."""
+    n_bags = bag_offsets.numel() - 1
+    K = len(worker_sample_offsets) - 1
+    _check(lib().antdt_embbag_bwd_dedup_static(
+        _dp(row_ids), row_ids.numel(), _dp(bag_offsets), n_bags, bags_per_sample, _dp(d_pooled),
+        d_pooled.shape[1], n_rows, K, _i64s(worker_sample_offsets), _dp(uniq_ids),
+        _dp(worker_uniq_offsets), _dp(seg_offsets), _dp(sorted_occ), _dp(uniq_grads),
+        uniq_grads.shape[0], _dp(dev_status), _stream(stream)), "antdt_embbag_bwd_dedup_static")
 
 
 def antdt_weighted_aggregate_workspace_bytes(in_cap: int, n_workers: int) -> int:
