@@ -141,6 +141,15 @@ def plan_all(w, n_steps):
     return plans
 
 
+def scaled_workload(w, scale):
+    if scale == 1.0:
+        return w
+    B_ = max(w.K * max(w.min_batch, 1), int(w.B * scale) // w.K * w.K)
+    V = max(w.F, int(w.V * scale) // w.F * w.F)
+    return w.scaled(B=B_, V=V, dense_n=int(w.dense_n * scale) // 4 * 4,
+                    name=f"{w.name} scaled x{scale:g}")
+
+
 def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
     """Bytes each kernel of the step has to move per launch (per step for the radix kernels'
     sum), from the counts of the batch: the gathers at full multiplicity, every output once."""
@@ -265,7 +274,7 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     B.lib()
     cfg = args.config
-    w = synth.WORKLOADS[cfg]
+    w = scaled_workload(synth.WORKLOADS[cfg], args.scale)
     if world > 1:
         w = w.scaled(seed=w.seed + 1000 * rank)           # independent replicas
     W, K_steps = args.warmup, args.steps
@@ -353,7 +362,10 @@ def run_ours(args):
     samples = sum_over_ranks(float(samples_local), dev)
 
     # ---- end to end through antdt_bsp_step_host, page-locked host buffers ---------------------
-    e2e = run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream)
+    if args.no_e2e:
+        e2e = {"ms": float("nan"), "samples": 0, "h2d": 0, "d2h": 0}
+    else:
+        e2e = run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream)
     e2e_ms = max_over_ranks(e2e["ms"], dev)
     e2e_samples = sum_over_ranks(float(e2e["samples"]), dev)
 
@@ -399,9 +411,10 @@ def run_ours(args):
                          "126 MB L2", "batches_rotated": n_batches,
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"]},
-        "e2e": {"value": e2e_samples / (e2e_ms * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                "ms_per_step": e2e_ms / K_steps},
+        "e2e": None if args.no_e2e else {
+            "value": e2e_samples / (e2e_ms * 1e-3), "unit": UNIT,
+            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+            "ms_per_step": e2e_ms / K_steps},
         "gpu_launches": launches,
         "roofline": roof,
         "step_algorithmic_GB": round(sb / 1e9, 3),
@@ -494,7 +507,7 @@ def run_reference(args):
         return
     from paper_2404_09679_b200 import synth
     cfg = args.config
-    w = synth.WORKLOADS[cfg]
+    w = scaled_workload(synth.WORKLOADS[cfg], args.scale)
     dev = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
     plans = plan_all(w, 1)
     bm = synth.BatchMaker(w, dev)
@@ -541,6 +554,10 @@ def main():
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--scale", type=float, default=1.0,
+                    help="shrink batch, table rows and dense vector by this factor (profiling "
+                         "captures on a small case); the JSON line says so")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
