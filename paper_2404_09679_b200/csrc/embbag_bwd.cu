@@ -61,7 +61,7 @@ bwd_prep_kernel(const int64_t* __restrict__ wso, int K, int F, const int64_t* __
   for (int w = tid; w <= K; w += blockDim.x) {
     const int64_t bag = wso[w] * (int64_t)F;  // host checked: 0 <= bag <= n_bags
     occ_bounds[w] = bag_offsets[bag];          // the sort setup clamps and orders these
-    if (w < K) worker_b[w] = (float)(wso[w + 1] - wso[w]);
+    if (w < K) worker_b[w] = 1.0f / (float)(wso[w + 1] - wso[w]);  // 1/b_w (inf for an empty worker: unused)
   }
 }
 
@@ -100,16 +100,22 @@ expand_bags_kernel(const int64_t* __restrict__ bag_offsets, int64_t n_bags, int6
 
 // ---------------------------------------------------------------------------------------
 // Tile reduction.  A group of G lanes (one 16-byte vector of the row per lane and VPL step)
-// walks kRedTile consecutive sorted occurrences, summing gathered d_pooled rows; a run that
-// starts and ends inside the tile is written out (divided by b_w), the pieces of runs that
-// cross the tile's edges go to head_part / tail_part for the fix-up pass.
+// walks kRedTile = 64 consecutive sorted occurrences, summing gathered d_pooled rows; a run that
+// starts and ends inside the tile is written out (times 1/b_w), the pieces of runs that cross
+// the tile's edges go to head_part / tail_part for the fix-up pass.
+//
+// The kernel is issue-bound once a worker's d_pooled slice sits in L2, so the walk is built to
+// cost few instructions per occurrence: the tile's run ends are one 64-bit mask consumed with
+// constant shifts, the bag indices of G occurrences live in one register per lane and are
+// broadcast by shuffle, kRedUnroll row loads are in flight before the first add, and the
+// worker (for the 1/b_w scale) is only re-resolved when the walk crosses a worker boundary.
 // ---------------------------------------------------------------------------------------
 template <int G, int VPL>
 __global__ void __launch_bounds__(kRedThreads)
 seg_reduce_tiles_kernel(const uint32_t* __restrict__ sorted_occ, const uint32_t* __restrict__ head_bits,
                         const int32_t* __restrict__ tile_first, const float* __restrict__ d_pooled,
                         int dim, int64_t n, int64_t n_bags, const int64_t* __restrict__ occ_bounds,
-                        const float* __restrict__ worker_b, int K, int64_t out_cap,
+                        const float* __restrict__ worker_inv, int K, int64_t out_cap,
                         float* __restrict__ uniq_grads, float* __restrict__ head_part,
                         float* __restrict__ tail_part) {
   extern __shared__ int64_t s_bounds[];  // [K+1]
@@ -119,79 +125,83 @@ seg_reduce_tiles_kernel(const uint32_t* __restrict__ sorted_occ, const uint32_t*
   const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
   const int64_t o_begin = tile * kRedTile;
   if (o_begin >= n) return;
-  const int64_t o_end = min(n, o_begin + kRedTile);
+  const int nv = (int)min((int64_t)kRedTile, n - o_begin);  // occurrences in this tile
   const unsigned gmask = group_mask<G>();
   const int nvec = dim / 4;
+  constexpr int U = (G < kRedUnroll) ? G : kRedUnroll;
 
-  // head flags of positions o_begin .. o_begin+kRedTile (one past the tile)
-  uint32_t hb[kRedTile / 32 + 1];
-#pragma unroll
-  for (int i = 0; i <= kRedTile / 32; ++i) hb[i] = __ldg(head_bits + (o_begin >> 5) + i);
-  auto is_head = [&](int rel) -> bool { return (hb[rel >> 5] >> (rel & 31)) & 1u; };
+  // run heads of positions o_begin .. o_begin+64; occurrence r closes its run iff r+1 is a head
+  const uint32_t* hw = head_bits + (o_begin >> 5);
+  const uint32_t h0 = __ldg(hw), h1 = __ldg(hw + 1), h2 = __ldg(hw + 2);
+  const uint64_t heads = (uint64_t)h0 | ((uint64_t)h1 << 32);
+  uint64_t ends = (heads >> 1) | ((uint64_t)(h2 & 1u) << 63);
+  const bool last_tile = o_begin + kRedTile >= n;
+  if (last_tile) ends = (ends & ((1ull << (nv - 1)) - 1ull)) | (1ull << (nv - 1));  // array end closes
+  const bool open_tail = !last_tile && !(h2 & 1u);  // the last run goes on in the next tile
 
   int64_t u = tile_first[tile];
-  bool started = is_head(0);
+  bool started = (h0 & 1u) != 0;
   int w = interval_of(s_bounds, K + 1, o_begin);
   if (w > K - 1) w = K - 1;
+  // tile-relative position at which the next worker starts (beyond the tile: never reached)
+  int next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
+  float inv = worker_inv[w];
 
   float4 acc[VPL];
 #pragma unroll
   for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  const uint32_t row_stride = (uint32_t)dim;
 
-  for (int64_t base = o_begin; base < o_end; base += G) {
-    const int cnt = (int)min((int64_t)G, o_end - base);
-    int64_t my_bag = -1;
-    if (lg < cnt) {
-      my_bag = (int64_t)__ldg(sorted_occ + base + lg);
-      if (my_bag >= n_bags) my_bag = -1;  // payload of a skipped (malformed) bag group
+  for (int q = 0; q * G < nv; ++q) {
+    int my_bag = -1;
+    if (q * G + lg < nv) {
+      const uint32_t bg = __ldg(sorted_occ + o_begin + q * G + lg);
+      my_bag = ((int64_t)bg < n_bags) ? (int)bg : -1;  // -1: payload of a skipped (malformed) bag
     }
-    for (int j = 0; j < cnt; j += kRedUnroll) {
-      float4 v[kRedUnroll][VPL];
-      bool ok[kRedUnroll];
 #pragma unroll
-      for (int t = 0; t < kRedUnroll; ++t) {
-        const int bag = (int)__shfl_sync(gmask, (int)my_bag, (j + t) & (G - 1), G);
-        ok[t] = (j + t < cnt) && bag >= 0;
-        if (ok[t]) {
-          const float* rp = d_pooled + (size_t)bag * dim;
+    for (int j0 = 0; j0 < G; j0 += U) {
+      float4 v[U][VPL];
 #pragma unroll
-          for (int k = 0; k < VPL; ++k) {
-            const int vi = lg + k * G;
-            if (vi < nvec) v[t][k] = ldg_f4(rp + 4 * vi);
-          }
+      for (int t = 0; t < U; ++t) {
+        const int bag = __shfl_sync(gmask, my_bag, j0 + t, G);
+        const float* rp = d_pooled + (size_t)((uint32_t)(bag < 0 ? 0 : bag)) * row_stride;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          const int vi = lg + k * G;
+          v[t][k] = (bag >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
       }
 #pragma unroll
-      for (int t = 0; t < kRedUnroll; ++t) {
-        if (j + t >= cnt) break;
-        if (ok[t]) {
+      for (int t = 0; t < U; ++t) {
 #pragma unroll
-          for (int k = 0; k < VPL; ++k) {
-            if (lg + k * G >= nvec) continue;
-            acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
-            acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
-          }
+        for (int k = 0; k < VPL; ++k) {
+          acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
+          acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
         }
-        const int64_t o = base + j + t;
-        const int rel = (int)(o - o_begin);
-        if (o + 1 == n || is_head(rel + 1)) {  // o closes its run
+        if ((ends >> (j0 + t)) & 1ull) {  // this occurrence closes its run
           float* dst;
-          float scale = 1.f;
+          float sc = 1.f;
           if (started) {
-            while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
-            scale = worker_b[w];
-            dst = (u < out_cap) ? uniq_grads + (size_t)u * dim : nullptr;
+            const int rel = q * G + j0 + t;
+            if (rel >= next_w_rel) {  // crossed into a later worker's range
+              const int64_t o = o_begin + rel;
+              while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
+              next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
+              if (w == K - 1) next_w_rel = kRedTile + 1;
+              inv = worker_inv[w];
+            }
+            sc = inv;
+            dst = (u < out_cap) ? uniq_grads + (size_t)u * row_stride : nullptr;
           } else {
-            dst = head_part + (size_t)tile * dim;
+            dst = head_part + (size_t)tile * row_stride;
           }
           if (dst) {
 #pragma unroll
             for (int k = 0; k < VPL; ++k) {
               const int vi = lg + k * G;
-              if (vi >= nvec) continue;
-              float4 r = acc[k];
-              if (started) { r.x /= scale; r.y /= scale; r.z /= scale; r.w /= scale; }
-              reinterpret_cast<float4*>(dst)[vi] = r;
+              if (vi < nvec)
+                reinterpret_cast<float4*>(dst)[vi] =
+                    make_float4(acc[k].x * sc, acc[k].y * sc, acc[k].z * sc, acc[k].w * sc);
             }
           }
           ++u;
@@ -201,10 +211,10 @@ seg_reduce_tiles_kernel(const uint32_t* __restrict__ sorted_occ, const uint32_t*
         }
       }
     }
+    ends = (G >= 64) ? 0ull : (ends >> (G & 63));
   }
-  // the run of the tile's last occurrence goes on in the next tile
-  if (o_end < n && !is_head((int)(o_end - o_begin))) {
-    float* dst = (started ? tail_part : head_part) + (size_t)tile * dim;
+  if (open_tail) {
+    float* dst = (started ? tail_part : head_part) + (size_t)tile * row_stride;
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
       const int vi = lg + k * G;
@@ -219,7 +229,7 @@ template <int G, int VPL>
 __global__ void __launch_bounds__(kRedThreads)
 seg_reduce_fixup_kernel(const uint32_t* __restrict__ head_bits, const int32_t* __restrict__ tile_first,
                         int dim, int64_t n, const int64_t* __restrict__ occ_bounds,
-                        const float* __restrict__ worker_b, int K, int64_t out_cap,
+                        const float* __restrict__ worker_inv, int K, int64_t out_cap,
                         float* __restrict__ uniq_grads, const float* __restrict__ head_part,
                         const float* __restrict__ tail_part) {
   const int lg = threadIdx.x & (G - 1);
@@ -266,14 +276,14 @@ seg_reduce_fixup_kernel(const uint32_t* __restrict__ head_bits, const int32_t* _
   // worker of the run = worker of any of its occurrences
   int w = interval_of(occ_bounds, K + 1, o_end - 1);
   if (w > K - 1) w = K - 1;
-  const float scale = worker_b[w];
+  const float scale = worker_inv[w];
   float* dst = uniq_grads + (size_t)u * dim;
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
     const int vi = lg + k * G;
     if (vi >= nvec) continue;
     float4 r = tot[k];
-    r.x /= scale; r.y /= scale; r.z /= scale; r.w /= scale;
+    r.x *= scale; r.y *= scale; r.z *= scale; r.w *= scale;
     reinterpret_cast<float4*>(dst)[vi] = r;
   }
 }
