@@ -64,7 +64,10 @@ segsort_setup_kernel(const int64_t* __restrict__ bounds_in, int S, int64_t n_cap
       prev = v;
     }
     const int64_t total = sb[S] - sb[0];
-    int64_t ce = (total + kSortChunksTarget - 1) / kSortChunksTarget;
+    // every segment ends in a partial chunk: aim for (slots - S) chunks so that all of them
+    // are resident at once (one wave at kSortCtasPerSM CTAs per SM)
+    const int64_t target = max(kSortChunksTarget / 2, kSortChunksTarget - S);
+    int64_t ce = (total + target - 1) / target;
     ce = ((ce + kSortTile - 1) / kSortTile) * kSortTile;
     if (ce < kSortTile) ce = kSortTile;
     s_chunk_elems = ce;
@@ -101,7 +104,27 @@ segsort_setup_kernel(const int64_t* __restrict__ bounds_in, int S, int64_t n_cap
 
 // ---------------------------------------------------------------------------------------
 // pass step 1: digit histogram of every chunk
+// Each thread takes 8 consecutive keys (two 16-byte loads where the run of 8 lies inside the
+// chunk) and adds run lengths, not single keys, to the shared histogram: after the first pass
+// equal keys sit together, so a hot row costs one shared-memory add per 8 keys instead of
+// serialising a warp on one counter.
 // ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void hist_add8(uint32_t* sh, const uint32_t (&k)[8], int shift, uint32_t mask) {
+  uint32_t cur = (k[0] >> shift) & mask, cnt = 1;
+#pragma unroll
+  for (int j = 1; j < 8; ++j) {
+    const uint32_t d = (k[j] >> shift) & mask;
+    if (d == cur) {
+      ++cnt;
+    } else {
+      atomicAdd(&sh[cur], cnt);
+      cur = d;
+      cnt = 1;
+    }
+  }
+  atomicAdd(&sh[cur], cnt);
+}
+
 __global__ void __launch_bounds__(kSortThreads)
 radix_hist_kernel(const uint32_t* __restrict__ keys, int shift, uint32_t mask,
                   const SortDesc* __restrict__ desc, const int64_t* __restrict__ chunk_begin,
@@ -110,25 +133,55 @@ radix_hist_kernel(const uint32_t* __restrict__ keys, int shift, uint32_t mask,
   const int c = blockIdx.x;
   if (c >= desc->n_chunks) return;
   __shared__ uint32_t sh[kSortMaxBins];
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x;
   for (int d = tid; d < kSortMaxBins; d += kSortThreads) sh[d] = 0;
   __syncthreads();
   const int64_t b = chunk_begin[c], e = chunk_end[c];
-  bool bad = false;
-  for (int64_t i0 = b; i0 < e; i0 += kSortThreads) {
-    const int64_t i = i0 + tid;
-    const bool valid = i < e;
-    uint32_t d = kSortMaxBins;  // sentinel: matches only other idle lanes
-    if (valid) {
-      const uint32_t k = __ldg(keys + i);
-      bad |= (check_rows > 0 && (int64_t)k >= check_rows);
-      d = (k >> shift) & mask;
+  const uint32_t limit = check_rows > 0 ? (uint32_t)check_rows : 0xffffffffu;
+  uint32_t kmax = 0;
+  // groups of 8 keys that start on a 16-byte boundary, whatever the array's own alignment
+  const int64_t off = (int64_t)((reinterpret_cast<uintptr_t>(keys) >> 2) & 3);
+  const int64_t ab = ((b + off) & ~(int64_t)7) - off;
+  constexpr int64_t kStep = (int64_t)kSortThreads * 8;
+  for (int64_t base = ab + (int64_t)tid * 8; base < e; base += 2 * kStep) {
+    const int64_t base2 = base + kStep;
+    const bool full1 = base >= b && base + 8 <= e;
+    const bool full2 = base2 >= b && base2 + 8 <= e;
+    uint4 x0, x1, y0, y1;
+    if (full1) {
+      x0 = __ldg(reinterpret_cast<const uint4*>(keys + base));
+      x1 = __ldg(reinterpret_cast<const uint4*>(keys + base) + 1);
     }
-    // one shared-memory add per distinct digit in the warp (hot rows would serialise otherwise)
-    const unsigned m = __match_any_sync(0xffffffffu, d);
-    if (valid && lane == __ffs(m) - 1) atomicAdd(&sh[d], (uint32_t)__popc(m));
+    if (full2) {
+      y0 = __ldg(reinterpret_cast<const uint4*>(keys + base2));
+      y1 = __ldg(reinterpret_cast<const uint4*>(keys + base2) + 1);
+    }
+    if (full1) {
+      const uint32_t k[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) kmax = max(kmax, k[j]);
+      hist_add8(sh, k, shift, mask);
+    } else {
+      for (int64_t i = max(base, b); i < min(base + 8, e); ++i) {
+        const uint32_t k = __ldg(keys + i);
+        kmax = max(kmax, k);
+        atomicAdd(&sh[(k >> shift) & mask], 1u);
+      }
+    }
+    if (full2) {
+      const uint32_t k[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) kmax = max(kmax, k[j]);
+      hist_add8(sh, k, shift, mask);
+    } else {
+      for (int64_t i = max(base2, b); i < min(base2 + 8, e); ++i) {
+        const uint32_t k = __ldg(keys + i);
+        kmax = max(kmax, k);
+        atomicAdd(&sh[(k >> shift) & mask], 1u);
+      }
+    }
   }
-  if (bad) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
+  if (kmax >= limit && check_rows > 0) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
   __syncthreads();
   for (int d = tid; d < kSortMaxBins; d += kSortThreads) hist[(size_t)c * kSortMaxBins + d] = sh[d];
 }
@@ -170,8 +223,17 @@ radix_scan_kernel(const SortDesc* __restrict__ desc, const int32_t* __restrict__
 
 // ---------------------------------------------------------------------------------------
 // pass step 3: stable scatter
+// 512 threads x 8 pairs per tile of 4096.  Phases per tile (a block barrier between each):
+// load -> rank inside the warp (match.any + per-warp counters) -> exclusive scan of the
+// counters over the warps and over the bins -> reorder the tile in shared memory -> write
+// every bin's run to its global slot with consecutive threads.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSortThreads)
+constexpr int kScatThreads = 512;
+constexpr int kScatItems = kSortTile / kScatThreads;  // 8
+constexpr int kScatWarps = kScatThreads / 32;         // 16
+constexpr size_t kScatSmem = 3 * kSortMaxBins * 4 + kScatWarps * kSortMaxBins * 2 + 2 * kSortTile * 4 + 64;
+
+__global__ void __launch_bounds__(kScatThreads, kSortCtasPerSM)
 radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
                      uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out, int shift,
                      uint32_t mask, const SortDesc* __restrict__ desc,
@@ -180,227 +242,252 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
                      const uint32_t* __restrict__ hist, const uint32_t* __restrict__ bin_base) {
   const int c = blockIdx.x;
   if (c >= desc->n_chunks) return;
-  constexpr int kWarps = kSortThreads / 32;
-  __shared__ uint32_t gbase[kSortMaxBins];      // next global slot of every bin (this chunk)
-  __shared__ uint32_t bin_start[kSortMaxBins];  // first slot of every bin inside the tile
-  __shared__ uint32_t bin_cnt[kSortMaxBins];
-  __shared__ unsigned short wh[kWarps][kSortMaxBins];
-  __shared__ uint32_t skeys[kSortTile];
-  __shared__ uint32_t svals[kSortTile];
-  __shared__ uint32_t warp_tot[kWarps];
+  extern __shared__ __align__(16) unsigned char scat_smem[];
+  uint32_t* gbase = reinterpret_cast<uint32_t*>(scat_smem);  // next global slot of every bin
+  uint32_t* bin_start = gbase + kSortMaxBins;                // first slot of every bin in the tile
+  uint32_t* bin_cnt = bin_start + kSortMaxBins;
+  uint32_t* skeys = bin_cnt + kSortMaxBins;
+  uint32_t* svals = skeys + kSortTile;
+  uint32_t* warp_tot = svals + kSortTile;                    // [16]
+  unsigned short* wh = reinterpret_cast<unsigned short*>(warp_tot + 16);  // [16][512]
 
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
   const unsigned lt = (1u << lane) - 1u;
   const int seg = chunk_seg[c];
   const uint32_t seg_begin = (uint32_t)seg_bounds[seg];
-  for (int d = tid; d < kSortMaxBins; d += kSortThreads)
-    gbase[d] = seg_begin + bin_base[(size_t)seg * kSortMaxBins + d] +
-               hist[(size_t)c * kSortMaxBins + d];
+  gbase[tid] = seg_begin + bin_base[(size_t)seg * kSortMaxBins + tid] + hist[(size_t)c * kSortMaxBins + tid];
+  unsigned short* my_wh = wh + w * kSortMaxBins;
 
   const int64_t cb = chunk_begin[c], ce = chunk_end[c];
   for (int64_t pos = cb; pos < ce; pos += kSortTile) {
     const int tile_n = (int)min((int64_t)kSortTile, ce - pos);
-    uint32_t k[kSortItems], v[kSortItems];
-    unsigned short rank[kSortItems];
-    // warp-striped: warp w owns elements [w*512, w*512+512) of the tile, item i of lane l is
-    // element w*512 + i*32 + l, so (item, lane) order is element order
-    const int wbase = w * (32 * kSortItems) + lane;
+    uint32_t k[kScatItems], v[kScatItems];
+    unsigned short rank[kScatItems];
+    // warp-striped: warp w owns elements [w*256, w*256+256) of the tile, item i of lane l is
+    // element w*256 + i*32 + l, so (item, lane) order is element order
+    const int wbase = w * (32 * kScatItems) + lane;
 #pragma unroll
-    for (int i = 0; i < kSortItems; ++i) {
+    for (int i = 0; i < kScatItems; ++i) {
       const int j = wbase + i * 32;
-      if (j < tile_n) {
-        k[i] = __ldg(keys_in + pos + j);
-        v[i] = vals_in ? __ldg(vals_in + pos + j) : (uint32_t)(pos + j);
-      } else {
-        k[i] = 0xffffffffu;
-        v[i] = 0;
-      }
+      const bool valid = j < tile_n;
+      k[i] = valid ? __ldg(keys_in + pos + j) : 0xffffffffu;
+      v[i] = valid ? (vals_in ? __ldg(vals_in + pos + j) : (uint32_t)(pos + j)) : 0u;
     }
-    uint32_t* whz = reinterpret_cast<uint32_t*>(&wh[0][0]);
-    for (int d = tid; d < kWarps * kSortMaxBins / 2; d += kSortThreads) whz[d] = 0;
+    {
+      uint32_t* whz = reinterpret_cast<uint32_t*>(wh);
+#pragma unroll
+      for (int d = 0; d < kScatWarps * kSortMaxBins / 2 / kScatThreads; ++d) whz[tid + d * kScatThreads] = 0;
+    }
     __syncthreads();  // (A) also: the previous tile's write-out is over
 
 #pragma unroll
-    for (int i = 0; i < kSortItems; ++i) {
+    for (int i = 0; i < kScatItems; ++i) {
       const bool valid = wbase + i * 32 < tile_n;
       const uint32_t d = valid ? ((k[i] >> shift) & mask) : (uint32_t)kSortMaxBins;
       const unsigned m = __match_any_sync(0xffffffffu, d);
-      const int leader = __ffs(m) - 1;
-      uint32_t old = 0;
-      if (valid && lane == leader) {
-        old = wh[w][d];
-        wh[w][d] = (unsigned short)(old + __popc(m));
-      }
-      old = __shfl_sync(0xffffffffu, old, leader);
-      rank[i] = (unsigned short)(old + __popc(m & lt));
+      // every peer reads the counter (one broadcast), the first peer then bumps it
+      const uint32_t old = valid ? my_wh[d] : 0u;
       __syncwarp();
+      if (valid && (m & lt) == 0) my_wh[d] = (unsigned short)(old + __popc(m));
+      __syncwarp();
+      rank[i] = (unsigned short)(old + __popc(m & lt));
     }
     __syncthreads();  // (B)
 
-    // per bin: exclusive scan over the warps; bin totals
-    for (int d = tid; d < kSortMaxBins; d += kSortThreads) {
-      uint32_t s = 0;
+    {  // per bin (one per thread): exclusive scan over the warps; bin totals
+      uint32_t sum = 0;
 #pragma unroll
-      for (int ww = 0; ww < kWarps; ++ww) {
-        const uint32_t t = wh[ww][d];
-        wh[ww][d] = (unsigned short)s;
-        s += t;
+      for (int ww = 0; ww < kScatWarps; ++ww) {
+        const uint32_t t = wh[ww * kSortMaxBins + tid];
+        wh[ww * kSortMaxBins + tid] = (unsigned short)sum;
+        sum += t;
       }
-      bin_cnt[d] = s;
-    }
-    __syncthreads();  // (C)
-
-    {  // exclusive scan over the 512 bins: thread t owns bins 2t and 2t+1
-      const uint32_t a = bin_cnt[2 * tid], b2 = bin_cnt[2 * tid + 1];
-      uint32_t incl = a + b2;
+      bin_cnt[tid] = sum;
+      // exclusive scan over the 512 bins
+      uint32_t incl = sum;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += t;
       }
       if (lane == 31) warp_tot[w] = incl;
-      __syncthreads();
+      __syncthreads();  // (C)
       uint32_t wp = 0;
 #pragma unroll
-      for (int ww = 0; ww < kWarps; ++ww) wp += (ww < w) ? warp_tot[ww] : 0u;
-      const uint32_t excl = incl - (a + b2) + wp;
-      bin_start[2 * tid] = excl;
-      bin_start[2 * tid + 1] = excl + a;
+      for (int ww = 0; ww < kScatWarps; ++ww) wp += (ww < w) ? warp_tot[ww] : 0u;
+      bin_start[tid] = incl - sum + wp;
     }
     __syncthreads();  // (D)
 
 #pragma unroll
-    for (int i = 0; i < kSortItems; ++i) {
+    for (int i = 0; i < kScatItems; ++i) {
       if (wbase + i * 32 < tile_n) {
         const uint32_t d = (k[i] >> shift) & mask;
-        const uint32_t p = bin_start[d] + wh[w][d] + rank[i];
+        const uint32_t p = bin_start[d] + my_wh[d] + rank[i];
         skeys[p] = k[i];
         svals[p] = v[i];
       }
     }
     __syncthreads();  // (E)
 
-    for (int j = tid; j < tile_n; j += kSortThreads) {
-      const uint32_t kk = skeys[j];
-      const uint32_t d = (kk >> shift) & mask;
-      const uint32_t g = gbase[d] + ((uint32_t)j - bin_start[d]);
-      keys_out[g] = kk;
-      vals_out[g] = svals[j];
+#pragma unroll
+    for (int i = 0; i < kScatItems; ++i) {
+      const int j = tid + i * kScatThreads;
+      if (j < tile_n) {
+        const uint32_t kk = skeys[j];
+        const uint32_t d = (kk >> shift) & mask;
+        const uint32_t g = gbase[d] + ((uint32_t)j - bin_start[d]);
+        keys_out[g] = kk;
+        vals_out[g] = svals[j];
+      }
     }
     __syncthreads();  // (F)
-    for (int d = tid; d < kSortMaxBins; d += kSortThreads) gbase[d] += bin_cnt[d];
+    gbase[tid] += bin_cnt[tid];
   }
 }
 
 // ---------------------------------------------------------------------------------------
 // runs of equal keys
+// A chunk is cut into kRunStrips 32-aligned strips, one warp each.  count: heads per strip;
+// scan: exclusive scan over all strips of all chunks; emit: every warp walks its strip once,
+// knowing how many runs start before it.  No block barrier inside the walks; 8 x 32 keys are
+// loaded before the first is used.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSortThreads)
+constexpr int kRunThreads = 512;
+constexpr int kRunStrips = kRunThreads / 32;  // 16
+constexpr int kRunUnroll = 8;
+
+struct Strip { int64_t s0, lo, hi; };  // aligned start, clipped [lo, hi)
+
+__device__ __forceinline__ Strip strip_of(int64_t b, int64_t e, int w) {
+  const int64_t ab = b & ~(int64_t)31;
+  const int64_t len = (((e - ab) + kRunStrips - 1) / kRunStrips + 31) & ~(int64_t)31;
+  Strip st;
+  st.s0 = ab + (int64_t)w * len;
+  st.lo = max(st.s0, b);
+  st.hi = min(e, st.s0 + len);
+  return st;
+}
+
+// head flags of the 32 elements [i0, i0+32) of a strip; key = this lane's key (if in range)
+__device__ __forceinline__ bool head_at(const uint32_t* __restrict__ keys, int64_t i, const Strip& st,
+                                        int64_t seg_begin, uint32_t key, uint32_t prev_lane_key,
+                                        int lane) {
+  if (i < st.lo || i >= st.hi) return false;
+  if (i == seg_begin) return true;
+  const uint32_t prev = (lane == 0 || i == st.lo) ? __ldg(keys + i - 1) : prev_lane_key;
+  return key != prev;
+}
+
+__global__ void __launch_bounds__(kRunThreads)
 runs_count_kernel(const uint32_t* __restrict__ keys, const SortDesc* __restrict__ desc,
                   const int32_t* __restrict__ chunk_seg, const int64_t* __restrict__ seg_bounds,
                   const int64_t* __restrict__ chunk_begin, const int64_t* __restrict__ chunk_end,
-                  int64_t* __restrict__ chunk_runs) {
+                  int64_t* __restrict__ strip_runs) {
   const int c = blockIdx.x;
   if (c >= desc->n_chunks) return;
-  const int tid = threadIdx.x;
-  const int64_t b = chunk_begin[c], e = chunk_end[c];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const Strip st = strip_of(chunk_begin[c], chunk_end[c], w);
   const int64_t seg_begin = seg_bounds[chunk_seg[c]];
   int cnt = 0;
-  for (int64_t i = b + tid; i < e; i += kSortThreads)
-    cnt += (i == seg_begin) || (__ldg(keys + i) != __ldg(keys + i - 1));
-  __shared__ int wsum[kSortThreads / 32];
+  for (int64_t j0 = st.s0; j0 < st.hi; j0 += 32 * kRunUnroll) {
+    uint32_t k[kRunUnroll];
+#pragma unroll
+    for (int r = 0; r < kRunUnroll; ++r) {
+      const int64_t i = j0 + r * 32 + lane;
+      k[r] = (i >= st.lo && i < st.hi) ? __ldg(keys + i) : 0u;
+    }
+#pragma unroll
+    for (int r = 0; r < kRunUnroll; ++r) {
+      const int64_t i = j0 + r * 32 + lane;
+      const uint32_t pk = __shfl_up_sync(0xffffffffu, k[r], 1);
+      cnt += head_at(keys, i, st, seg_begin, k[r], pk, lane) ? 1 : 0;
+    }
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, o);
-  if ((tid & 31) == 0) wsum[tid >> 5] = cnt;
-  __syncthreads();
-  if (tid == 0) {
-    int t = 0;
-    for (int ww = 0; ww < kSortThreads / 32; ++ww) t += wsum[ww];
-    chunk_runs[c] = t;
-  }
+  if (lane == 0) strip_runs[(size_t)c * kRunStrips + w] = cnt;
 }
 
 __global__ void __launch_bounds__(1024)
 runs_scan_kernel(const SortDesc* __restrict__ desc, const int32_t* __restrict__ seg_first,
-                 int64_t* chunk_runs, int64_t* seg_runs, int64_t* n_runs_out, int64_t* run_start,
+                 int64_t* strip_runs, int64_t* seg_runs, int64_t* n_runs_out, int64_t* run_start,
                  int64_t out_cap, int32_t* status) {
   __shared__ int64_t warp_tot[32];
   __shared__ int64_t total;
-  const int n_chunks = desc->n_chunks;
+  const int n = desc->n_chunks * kRunStrips;
   const int tid = threadIdx.x;
-  const int per = (n_chunks + 1023) / 1024;  // consecutive chunks per thread
-  const int c0 = tid * per, c1 = min(n_chunks, c0 + per);
+  const int per = (n + 1023) / 1024;  // consecutive strips per thread
+  const int c0 = tid * per, c1 = min(n, c0 + per);
   int64_t mine = 0;
-  for (int c = c0; c < c1; ++c) mine += chunk_runs[c];
+  for (int c = c0; c < c1; ++c) mine += strip_runs[c];
   int64_t excl = block_exclusive_scan_1024(mine, &total, warp_tot);
   for (int c = c0; c < c1; ++c) {
-    const int64_t t = chunk_runs[c];
-    chunk_runs[c] = excl;
+    const int64_t t = strip_runs[c];
+    strip_runs[c] = excl;
     excl += t;
   }
   __syncthreads();
   if (tid == 0) {
-    chunk_runs[n_chunks] = total;
+    strip_runs[n] = total;
     if (n_runs_out) *n_runs_out = total;
     run_start[total < out_cap ? total : out_cap] = desc->n;
     if (total > out_cap) set_status(status, ANTDT_ERR_CAPACITY);
   }
   __syncthreads();
   if (seg_runs)
-    for (int s = tid; s <= desc->n_segments; s += blockDim.x) seg_runs[s] = chunk_runs[seg_first[s]];
+    for (int s = tid; s <= desc->n_segments; s += blockDim.x)
+      seg_runs[s] = strip_runs[(size_t)seg_first[s] * kRunStrips];
 }
 
-__global__ void __launch_bounds__(kSortThreads)
+__global__ void __launch_bounds__(kRunThreads)
 runs_emit_kernel(const uint32_t* __restrict__ keys, const SortDesc* __restrict__ desc,
                  const int32_t* __restrict__ chunk_seg, const int64_t* __restrict__ seg_bounds,
                  const int64_t* __restrict__ chunk_begin, const int64_t* __restrict__ chunk_end,
-                 const int64_t* __restrict__ chunk_runs, int32_t* __restrict__ uniq_keys,
+                 const int64_t* __restrict__ strip_runs, int32_t* __restrict__ uniq_keys,
                  int64_t* __restrict__ run_start, int64_t out_cap, uint32_t* head_bits,
-                 int32_t* __restrict__ tile_first, int tile) {
+                 int32_t* __restrict__ tile_first, int tile_shift) {
   const int c = blockIdx.x;
   if (c >= desc->n_chunks) return;
-  constexpr int kWarps = kSortThreads / 32;
-  __shared__ int wtot[kWarps];
-  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int64_t b = chunk_begin[c], e = chunk_end[c];
+  const Strip st = strip_of(b, e, w);
   const int64_t seg_begin = seg_bounds[chunk_seg[c]];
-  int64_t running = chunk_runs[c];  // runs that start before this chunk
-  for (int64_t i0 = b; i0 < e; i0 += kSortThreads) {
-    const int64_t i = i0 + tid;
-    const bool valid = i < e;
-    uint32_t key = 0;
-    bool head = false;
-    if (valid) {
-      key = __ldg(keys + i);
-      head = (i == seg_begin) || (key != __ldg(keys + i - 1));
-    }
-    const unsigned bal = __ballot_sync(0xffffffffu, head);
-    if (lane == 0) wtot[w] = __popc(bal);
-    __syncthreads();
-    int before = 0, all = 0;
+  const int64_t tile_mask = ((int64_t)1 << tile_shift) - 1;
+  int64_t running = strip_runs[(size_t)c * kRunStrips + w];  // runs that start before this strip
+  for (int64_t j0 = st.s0; j0 < st.hi; j0 += 32 * kRunUnroll) {
+    uint32_t k[kRunUnroll];
 #pragma unroll
-    for (int ww = 0; ww < kWarps; ++ww) {
-      const int t = wtot[ww];
-      before += ww < w ? t : 0;
-      all += t;
+    for (int r = 0; r < kRunUnroll; ++r) {
+      const int64_t i = j0 + r * 32 + lane;
+      k[r] = (i >= st.lo && i < st.hi) ? __ldg(keys + i) : 0u;
     }
-    const int64_t incl = running + before + __popc(bal & ((2u << lane) - 1u));
-    if (head) {
-      const int64_t r = incl - 1;
-      if (r < out_cap) {
-        uniq_keys[r] = (int32_t)key;
-        run_start[r] = i;
+#pragma unroll
+    for (int r = 0; r < kRunUnroll; ++r) {
+      const int64_t i0 = j0 + r * 32;
+      if (i0 >= st.hi) break;
+      const int64_t i = i0 + lane;
+      const uint32_t pk = __shfl_up_sync(0xffffffffu, k[r], 1);
+      const bool head = head_at(keys, i, st, seg_begin, k[r], pk, lane);
+      const unsigned bal = __ballot_sync(0xffffffffu, head);
+      const int64_t incl = running + __popc(bal & ((2u << lane) - 1u));
+      if (head) {
+        const int64_t rr = incl - 1;
+        if (rr < out_cap) {
+          uniq_keys[rr] = (int32_t)k[r];
+          run_start[rr] = i;
+        }
       }
+      if (tile_first && i >= st.lo && i < st.hi && (i & tile_mask) == 0)
+        tile_first[i >> tile_shift] = (int32_t)(incl - 1);
+      if (head_bits && lane == 0 && bal) {
+        // i0 is a multiple of 32: the ballot is exactly one word; words shared with another
+        // chunk (first / last word of the chunk) are merged with an atomic OR
+        if (i0 >= b && i0 + 32 <= e) head_bits[i0 >> 5] = bal;
+        else atomicOr(&head_bits[i0 >> 5], bal);
+      }
+      running += __popc(bal);
     }
-    if (valid && tile_first && (i % tile) == 0) tile_first[i / tile] = (int32_t)(incl - 1);
-    if (head_bits && lane == 0 && bal) {  // the warp's 32 flags straddle at most two words
-      const int64_t first = i0 + w * 32;
-      const int sh = (int)(first & 31);
-      atomicOr(&head_bits[first >> 5], bal << sh);
-      if (sh && (bal >> (32 - sh))) atomicOr(&head_bits[(first >> 5) + 1], bal >> (32 - sh));
-    }
-    running += all;
-    __syncthreads();
   }
 }
 
@@ -420,7 +507,7 @@ SortLayout sort_layout(int S) {
   L.chunk_end = o;   o = align_up(o + 8 * C);
   L.hist = o;        o = align_up(o + 4 * C * kSortMaxBins);
   L.bin_base = o;    o = align_up(o + 4 * (size_t)S * kSortMaxBins);
-  L.chunk_runs = o;  o = align_up(o + 8 * (C + 1));
+  L.chunk_runs = o;  o = align_up(o + 8 * (C * 16 + 1));
   L.bytes = o;
   return L;
 }
@@ -446,6 +533,14 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
   uint32_t* hist = (uint32_t*)(ws + L.hist);
   uint32_t* bin_base = (uint32_t*)(ws + L.bin_base);
   const int P = sort_passes(key_bits);
+  static bool carveout_set = false;
+  if (!carveout_set) {  // 4 CTAs x 46 KB of shared memory per SM need the large carve-out
+    cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kScatSmem);
+    cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                         cudaSharedmemCarveoutMaxShared);
+    carveout_set = true;
+  }
   // spread the bits evenly over the passes
   int shift = 0;
   const uint32_t* kin = keys_in;
@@ -462,7 +557,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
                  mask, desc, chunk_begin, chunk_end, hist, p == 0 ? check_rows : (int64_t)0, status);
     ANTDT_LAUNCH("radix_scan", radix_scan_kernel, S, kSortMaxBins, 0, s, desc, seg_first, hist,
                  bin_base);
-    ANTDT_LAUNCH("radix_scatter", radix_scatter_kernel, L.max_chunks, kSortThreads, 0, s, kin, vin,
+    ANTDT_LAUNCH("radix_scatter", radix_scatter_kernel, L.max_chunks, kScatThreads, kScatSmem, s, kin, vin,
                  kout, vout, shift, mask, desc, chunk_seg, seg_bounds, chunk_begin, chunk_end, hist,
                  bin_base);
     kin = kout;
@@ -483,13 +578,15 @@ void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys
   const int64_t* chunk_end = (const int64_t*)(ws + L.chunk_end);
   int64_t* chunk_runs = (int64_t*)(ws + L.chunk_runs);
   if (head_bits) cudaMemsetAsync(head_bits, 0, head_bits_words(n_cap) * 4, s);
-  ANTDT_LAUNCH("runs_count", runs_count_kernel, L.max_chunks, kSortThreads, 0, s, sorted_keys,
+  int tile_shift = 0;
+  while ((1 << tile_shift) < tile) ++tile_shift;  // tile is a power of two
+  ANTDT_LAUNCH("runs_count", runs_count_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys,
                desc, chunk_seg, seg_bounds, chunk_begin, chunk_end, chunk_runs);
   ANTDT_LAUNCH("runs_scan", runs_scan_kernel, 1, 1024, 0, s, desc, seg_first, chunk_runs, seg_runs,
                n_runs_out, run_start, out_cap, status);
-  ANTDT_LAUNCH("runs_emit", runs_emit_kernel, L.max_chunks, kSortThreads, 0, s, sorted_keys, desc,
+  ANTDT_LAUNCH("runs_emit", runs_emit_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys, desc,
                chunk_seg, seg_bounds, chunk_begin, chunk_end, chunk_runs, uniq_keys, run_start,
-               out_cap, head_bits, tile_first, tile);
+               out_cap, head_bits, tile_first, tile_shift);
 }
 
 }  // namespace antdt

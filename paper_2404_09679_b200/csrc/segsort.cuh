@@ -16,7 +16,8 @@
 
 namespace antdt {
 
-constexpr int kSortChunksTarget = kNumSM * 4;  // work units of the sort: one CTA each
+constexpr int kSortCtasPerSM = 3;                            // scatter CTAs resident per SM
+constexpr int kSortChunksTarget = kNumSM * kSortCtasPerSM;  // work units of the sort: one CTA each
 constexpr int kSortThreads = 256;
 constexpr int kSortItems = 16;
 constexpr int kSortTile = kSortThreads * kSortItems;  // 4096 pairs staged in shared memory
@@ -43,7 +44,7 @@ struct SortLayout {
   size_t chunk_end;    // int64 [C]
   size_t hist;         // uint32 [C * 512]
   size_t bin_base;     // uint32 [S * 512]
-  size_t chunk_runs;   // int64 [C + 1]  run counts per chunk (runs pass)
+  size_t chunk_runs;   // int64 [16 C + 1]  run counts per strip of a chunk (runs pass)
   size_t bytes;        // total
   int max_chunks;      // C
 };
@@ -77,7 +78,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
 //   seg_runs   [S+1]        runs before each segment; [S] = n_runs  (may be nullptr)
 //   n_runs_out one int64    (may be nullptr)
 //   head_bits  [head_bits_words(n_cap)] bit i set iff element i starts a run (zeroed here)
-//   tile_first [n_cap/tile+1] run index of element t*tile (may be nullptr)
+//   tile_first [n_cap/tile+1] run index of element t*tile (may be nullptr); tile a power of 2
 // More runs than out_cap -> CAPACITY in status, the excess is not written.
 void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys,
                   int64_t* run_start, int64_t* seg_runs, int64_t* n_runs_out, int64_t out_cap,
