@@ -52,6 +52,27 @@ __device__ __forceinline__ float4 ldg_f4(const float* p) {
   return __ldg(reinterpret_cast<const float4*>(p));
 }
 
+// Packed pairs of fp32 in one 64-bit register: sm_100 adds / multiplies two lanes per
+// instruction (each lane rounded exactly like the scalar operation).
+__device__ __forceinline__ uint64_t f32x2_pack(uint32_t lo_bits, uint32_t hi_bits) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo_bits), "r"(hi_bits));
+  return r;
+}
+__device__ __forceinline__ uint64_t f32x2_add(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f32x2_mul(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ ulonglong2 ldg_u64x2(const void* p) {
+  return __ldg(reinterpret_cast<const ulonglong2*>(p));
+}
+
 // 8 bf16 (one 16-byte vector) widened to fp32; widening is exact.
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* f) {
   f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);

@@ -19,7 +19,9 @@ embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
                   const int32_t* __restrict__ row_ids, int64_t nnz,
                   const int64_t* __restrict__ bag_offsets, int64_t n_bags,
                   float* __restrict__ pooled, int32_t* status) {
-  constexpr int EPV = BF16 ? 8 : 4;  // elements per 16-byte vector
+  constexpr int EPV = BF16 ? 8 : 4;   // elements per 16-byte vector
+  constexpr int PAIRS = EPV / 2;      // packed fp32 pairs per vector
+  constexpr int U = (G < kFwdUnroll) ? G : kFwdUnroll;
   const int lg = threadIdx.x & (G - 1);
   const int64_t bag = (int64_t)blockIdx.x * (kFwdThreads / G) + (threadIdx.x / G);
   if (bag >= n_bags) return;
@@ -31,56 +33,55 @@ embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
     if (lg == 0) set_status(status, ANTDT_ERR_BAD_OFFSETS);
     end = begin = 0;
   }
+  const int len = (int)(end - begin);
+  const int32_t* ids = row_ids + begin;
+  const uint32_t limit = (uint32_t)n_rows;
 
-  float acc[VPL][EPV];
+  uint64_t acc[VPL][PAIRS];  // fp32 sums as packed pairs
 #pragma unroll
   for (int k = 0; k < VPL; ++k)
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) acc[k][e] = 0.f;
+    for (int e = 0; e < PAIRS; ++e) acc[k][e] = 0ull;
 
   const char* tbl = static_cast<const char*>(table);
-  const size_t row_bytes = (size_t)dim * (BF16 ? 2 : 4);
+  const uint32_t row_bytes = (uint32_t)dim * (BF16 ? 2u : 4u);
 
-  for (int64_t base = begin; base < end; base += G) {
-    const int cnt = (int)min((int64_t)G, end - base);
-    int my_id = (lg < cnt) ? __ldg(row_ids + base + lg) : -1;
-    if (lg < cnt && (my_id < 0 || (int64_t)my_id >= n_rows)) {
-      set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
-      my_id = -1;  // skipped: contributes nothing
+  for (int base = 0; base < len; base += G) {
+    // G ids of the bag in one coalesced load; -1 marks "no row" (past the end, or out of range)
+    int my_id = -1;
+    if (base + lg < len) {
+      my_id = __ldg(ids + base + lg);
+      if ((uint32_t)my_id >= limit) {
+        set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
+        my_id = -1;  // skipped: contributes nothing
+      }
     }
-    for (int j = 0; j < cnt; j += kFwdUnroll) {
-      uint4 v[kFwdUnroll][VPL];
-      bool ok[kFwdUnroll];
 #pragma unroll
-      for (int u = 0; u < kFwdUnroll; ++u) {
-        // source lane stays inside the group even when j+u runs past cnt (id -1 there)
-        const int id = __shfl_sync(gmask, my_id, (j + u) & (G - 1), G);
-        ok[u] = (j + u < cnt) && id >= 0;
-        if (ok[u]) {
-          const uint4* rp = reinterpret_cast<const uint4*>(tbl + (size_t)id * row_bytes);
+    for (int j0 = 0; j0 < G; j0 += U) {
+      if (base + j0 >= len) break;
+      uint4 v[U][VPL];
 #pragma unroll
-          for (int k = 0; k < VPL; ++k) {
-            const int vi = lg + k * G;
-            if (vi < nvec) v[u][k] = __ldg(rp + vi);
-          }
+      for (int u = 0; u < U; ++u) {
+        const int id = __shfl_sync(gmask, my_id, j0 + u, G);
+        const uint4* rp = reinterpret_cast<const uint4*>(tbl + (size_t)(uint32_t)(id < 0 ? 0 : id) * row_bytes);
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          const int vi = lg + k * G;
+          v[u][k] = (id >= 0 && vi < nvec) ? __ldg(rp + vi) : make_uint4(0u, 0u, 0u, 0u);
         }
       }
 #pragma unroll
-      for (int u = 0; u < kFwdUnroll; ++u) {
-        if (!ok[u]) continue;
+      for (int u = 0; u < U; ++u) {
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-          if (lg + k * G >= nvec) continue;
-          if (BF16) {
-            float f[8];
-            bf16x8_to_f32(v[u][k], f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[k][e] += f[e];
+          if (BF16) {  // bf16 -> fp32 is a 16-bit shift; a zero vector adds +0.0
+            acc[k][0] = f32x2_add(acc[k][0], f32x2_pack(v[u][k].x << 16, v[u][k].x & 0xffff0000u));
+            acc[k][1] = f32x2_add(acc[k][1], f32x2_pack(v[u][k].y << 16, v[u][k].y & 0xffff0000u));
+            acc[k][2] = f32x2_add(acc[k][2], f32x2_pack(v[u][k].z << 16, v[u][k].z & 0xffff0000u));
+            acc[k][3] = f32x2_add(acc[k][3], f32x2_pack(v[u][k].w << 16, v[u][k].w & 0xffff0000u));
           } else {
-            acc[k][0] += __uint_as_float(v[u][k].x);
-            acc[k][1] += __uint_as_float(v[u][k].y);
-            acc[k][2] += __uint_as_float(v[u][k].z);
-            acc[k][3] += __uint_as_float(v[u][k].w);
+            acc[k][0] = f32x2_add(acc[k][0], f32x2_pack(v[u][k].x, v[u][k].y));
+            acc[k][1] = f32x2_add(acc[k][1], f32x2_pack(v[u][k].z, v[u][k].w));
           }
         }
       }
@@ -92,9 +93,9 @@ embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
   for (int k = 0; k < VPL; ++k) {
     const int vi = lg + k * G;
     if (vi >= nvec) continue;
-    float4* o = reinterpret_cast<float4*>(out + (size_t)vi * EPV);
-    o[0] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
-    if (BF16) o[1] = make_float4(acc[k][4], acc[k][5], acc[k][6], acc[k][7]);
+    ulonglong2* o = reinterpret_cast<ulonglong2*>(out + (size_t)vi * EPV);
+    o[0] = make_ulonglong2(acc[k][0], acc[k][1]);
+    if (BF16) o[1] = make_ulonglong2(acc[k][2], acc[k][3]);
   }
 }
 
