@@ -242,7 +242,7 @@ typedef struct {
   float* out;         /* device out [n]                                                   */
 } antdt_dense_part;
 
-size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32_t n_workers);
+size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32_t dim, int32_t n_workers);
 int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,
                                  const int64_t* batch_sizes, int32_t n_workers, void* ws,
                                  size_t ws_bytes, int32_t* dev_status, void* stream);

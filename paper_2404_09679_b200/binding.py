@@ -111,7 +111,7 @@ def lib() -> C.CDLL:
         L.antdt_embbag_bwd_dedup_static.argtypes = [P, I64, P, I64, I32, P, I32, I64, I32, P, P, P, P,
                                                     P, P, I64, P, P]
         L.antdt_embbag_bwd_dedup_static.restype = I32
-        L.antdt_weighted_aggregate_workspace_bytes.argtypes = [I64, I32]
+        L.antdt_weighted_aggregate_workspace_bytes.argtypes = [I64, I32, I32]
         L.antdt_weighted_aggregate_workspace_bytes.restype = SZ
         L.antdt_weighted_aggregate.argtypes = [P, P, P, I32, P, SZ, P, P]
         L.antdt_sparse_opt_update.argtypes = [P, I32, I64, I32, P, P, P, I64, I32, F, F, F, F, I64,
@@ -287,8 +287,8 @@ def antdt_embbag_bwd_dedup_static(row_ids, bag_offsets, bags_per_sample: int, d_
         uniq_grads.shape[0], _dp(dev_status), _stream(stream)), "antdt_embbag_bwd_dedup_static")
 
 
-def antdt_weighted_aggregate_workspace_bytes(in_cap: int, n_workers: int) -> int:
-    return lib().antdt_weighted_aggregate_workspace_bytes(in_cap, n_workers)
+def antdt_weighted_aggregate_workspace_bytes(in_cap: int, dim: int, n_workers: int) -> int:
+    return lib().antdt_weighted_aggregate_workspace_bytes(in_cap, dim, n_workers)
 
 
 def antdt_weighted_aggregate(batch_sizes: Sequence[int], ws, *, n_rows: int = 0, uniq_ids=None,

@@ -2,26 +2,26 @@
 //
 // Sparse part: the workers' row lists (each ascending) are merged by one stable radix sort of
 // (row id, position in the concatenated list); equal rows then sit together in ascending
-// worker order, so one group per output row sums its <= K weighted contributions in a fixed
-// order.  Because the sorted positions of one worker ascend with the row id, the gather of the
-// workers' gradient rows is K forward-moving streams, not a random walk.
+// worker order, and the tile-parallel segmented reduction (tile_reduce.cuh) forms each row's
+// weighted sum of its <= K contributions in that fixed order.  Because the sorted positions of
+// one worker ascend with the row id, the gather of the workers' gradient rows is K
+// forward-moving streams, not a random walk.
 // Dense part: a K-way streaming reduction, one 16-byte vector per thread and worker.
 #include "segsort.cuh"
+#include "tile_reduce.cuh"
 
 namespace antdt {
 namespace {
-
-constexpr int kAggThreads = 256;
-constexpr int kAggUnroll = 4;
 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct AggLayout {
   SortLayout sort;
-  size_t sort_ws, bounds, weights, wuo, keys_a, keys_b, src, vals_t, run_start, bytes;
+  size_t sort_ws, bounds, weights, wuo, keys_a, keys_b, src, vals_t, run_start, head_bits,
+      tile_first, head_part, tail_part, bytes;
 };
 
-AggLayout agg_layout(int64_t in_cap, int K) {
+AggLayout agg_layout(int64_t in_cap, int K, int dim) {
   AggLayout L;
   L.sort = sort_layout(1);
   const size_t n = (size_t)(in_cap > 0 ? in_cap : 1);
@@ -35,6 +35,11 @@ AggLayout agg_layout(int64_t in_cap, int K) {
   L.src = o;       o = align_up(o + 4 * n);
   L.vals_t = o;    o = align_up(o + 4 * n);
   L.run_start = o; o = align_up(o + 8 * (n + 1));
+  const size_t n_tiles = (n + kRedTile - 1) / kRedTile;
+  L.head_bits = o;  o = align_up(o + 4 * head_bits_words((int64_t)n));
+  L.tile_first = o; o = align_up(o + 4 * (n_tiles + 1));
+  L.head_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
+  L.tail_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
   L.bytes = o;
   return L;
 }
@@ -58,68 +63,6 @@ __global__ void agg_prep_kernel(const int64_t* __restrict__ wuo_in, int K, int64
     }
     bounds[0] = 0;
     bounds[1] = n;
-  }
-}
-
-// One group of G lanes per output row; grid-stride because the row count lives on the device.
-template <int G, int VPL>
-__global__ void __launch_bounds__(kAggThreads)
-agg_reduce_kernel(const int64_t* __restrict__ n_agg, int64_t out_cap,
-                  const int64_t* __restrict__ run_start, const uint32_t* __restrict__ src,
-                  const int64_t* __restrict__ wuo, const float* __restrict__ weights, int K,
-                  const float* __restrict__ uniq_grads, int dim, float* __restrict__ agg_grads) {
-  extern __shared__ int64_t s_wuo[];  // [K+1], then K floats
-  float* s_w = reinterpret_cast<float*>(s_wuo + (K + 1));
-  for (int i = threadIdx.x; i <= K; i += blockDim.x) s_wuo[i] = wuo[i];
-  for (int i = threadIdx.x; i < K; i += blockDim.x) s_w[i] = weights[i];
-  __syncthreads();
-  const int lg = threadIdx.x & (G - 1);
-  const int nvec = dim / 4;
-  const int64_t n = min(*n_agg, out_cap);
-  const int64_t stride = (int64_t)gridDim.x * (kAggThreads / G);
-  for (int64_t u = (int64_t)blockIdx.x * (kAggThreads / G) + threadIdx.x / G; u < n; u += stride) {
-    const int64_t b = run_start[u], e = run_start[u + 1];
-    float4 acc[VPL];
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int64_t j = b; j < e; j += kAggUnroll) {
-      float4 v[kAggUnroll][VPL];
-      float wt[kAggUnroll];
-#pragma unroll
-      for (int t = 0; t < kAggUnroll; ++t) {
-        wt[t] = 0.f;
-        if (j + t < e) {
-          const int64_t p = (int64_t)__ldg(src + j + t);  // same address for the whole group
-          int w = interval_of(s_wuo, K + 1, p);
-          if (w > K - 1) w = K - 1;
-          wt[t] = s_w[w];
-          const float* rp = uniq_grads + (size_t)p * dim;
-#pragma unroll
-          for (int k = 0; k < VPL; ++k) {
-            const int vi = lg + k * G;
-            if (vi < nvec) v[t][k] = ldg_f4(rp + 4 * vi);
-          }
-        }
-      }
-#pragma unroll
-      for (int t = 0; t < kAggUnroll; ++t) {
-        if (j + t >= e) break;
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-          if (lg + k * G >= nvec) continue;
-          acc[k].x = fmaf(wt[t], v[t][k].x, acc[k].x);
-          acc[k].y = fmaf(wt[t], v[t][k].y, acc[k].y);
-          acc[k].z = fmaf(wt[t], v[t][k].z, acc[k].z);
-          acc[k].w = fmaf(wt[t], v[t][k].w, acc[k].w);
-        }
-      }
-    }
-    float* dst = agg_grads + (size_t)u * dim;
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-      const int vi = lg + k * G;
-      if (vi < nvec) reinterpret_cast<float4*>(dst)[vi] = acc[k];
-    }
   }
 }
 
@@ -156,26 +99,14 @@ dense_wsum_kernel(const float* __restrict__ grads, int64_t n4, int64_t stride,
   }
 }
 
-template <int G, int VPL>
-void launch_agg_reduce(const antdt_sparse_part* sp, const AggLayout& L, char* ws, int K,
-                       cudaStream_t s) {
-  const int64_t gpb = kAggThreads / G;
-  int64_t want = (sp->out_cap + gpb - 1) / gpb;
-  const int64_t cap = (int64_t)kNumSM * 16;
-  const unsigned grid = (unsigned)(want < 1 ? 1 : (want > cap ? cap : want));
-  const size_t smem = 8 * ((size_t)K + 1) + 4 * (size_t)K;
-  ANTDT_LAUNCH("agg_reduce", (agg_reduce_kernel<G, VPL>), grid, kAggThreads, smem, s, sp->n_agg,
-               sp->out_cap, (const int64_t*)(ws + L.run_start), (const uint32_t*)(ws + L.src),
-               (const int64_t*)(ws + L.wuo), (const float*)(ws + L.weights), K, sp->uniq_grads,
-               (int)sp->dim, sp->agg_grads);
-}
-
 }  // namespace
 }  // namespace antdt
 
-extern "C" size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32_t n_workers) {
-  if (in_cap < 0 || n_workers < 1 || n_workers > antdt::kMaxSegments) return 0;
-  return antdt::agg_layout(in_cap, n_workers).bytes;
+extern "C" size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32_t dim,
+                                                           int32_t n_workers) {
+  if (in_cap < 0 || dim < 0 || dim > 1024 || n_workers < 1 || n_workers > antdt::kMaxSegments)
+    return 0;
+  return antdt::agg_layout(in_cap, n_workers, dim).bytes;
 }
 
 extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,
@@ -205,7 +136,7 @@ extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const a
     if (dp->n > 0 && (!dp->grads || !dp->out || !aligned16(dp->grads) || !aligned16(dp->out)))
       return ANTDT_ERR_INVALID_ARG;
   }
-  const AggLayout L = agg_layout(in_cap, K);
+  const AggLayout L = agg_layout(in_cap, K, sp ? sp->dim : 0);
   if (ws_bytes < L.bytes) return ANTDT_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t s = (cudaStream_t)stream;
   char* w8 = static_cast<char*>(ws);
@@ -226,20 +157,27 @@ extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const a
                 (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b), (uint32_t*)(w8 + L.vals_t),
                 bits_for(sp->n_rows), 0, sort_ws, L.sort, dev_status, s);
     segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
-                 sp->out_cap < in_cap ? sp->out_cap : in_cap, nullptr, nullptr, 1, sort_ws, L.sort,
-                 dev_status, s);
-    const int nvec = sp->dim / 4;
-#define AGG_CASE(G, VPL) launch_agg_reduce<G, VPL>(sp, L, w8, K, s);
-    if (nvec <= 1) { AGG_CASE(1, 1) }
-    else if (nvec <= 2) { AGG_CASE(2, 1) }
-    else if (nvec <= 4) { AGG_CASE(4, 1) }
-    else if (nvec <= 8) { AGG_CASE(8, 1) }
-    else if (nvec <= 16) { AGG_CASE(16, 1) }
-    else if (nvec <= 32) { AGG_CASE(32, 1) }
-    else if (nvec <= 64) { AGG_CASE(32, 2) }
-    else if (nvec <= 128) { AGG_CASE(32, 4) }
-    else { AGG_CASE(32, 8) }
-#undef AGG_CASE
+                 sp->out_cap < in_cap ? sp->out_cap : in_cap, (uint32_t*)(w8 + L.head_bits),
+                 (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s);
+    if (in_cap > 0) {
+      TileArgs t;
+      t.payload = (const uint32_t*)(w8 + L.src);
+      t.head_bits = (const uint32_t*)(w8 + L.head_bits);
+      t.tile_first = (const int32_t*)(w8 + L.tile_first);
+      t.rows = sp->uniq_grads;
+      t.dim = sp->dim;
+      t.n_host = in_cap;
+      t.n_dev = bounds + 1;  // the clamped total of the workers' lists
+      t.payload_limit = in_cap;
+      t.bounds = (const int64_t*)(w8 + L.wuo);
+      t.scales = (const float*)(w8 + L.weights);
+      t.K = K;
+      t.out_cap = sp->out_cap < in_cap ? sp->out_cap : in_cap;
+      t.out = sp->agg_grads;
+      t.head_part = (float*)(w8 + L.head_part);
+      t.tail_part = (float*)(w8 + L.tail_part);
+      launch_tile_reduce<true>(t, "agg_reduce", "agg_fixup", s);
+    }
   }
   if (dp && dp->n > 0) {
     const int64_t n4 = dp->n / 4;

@@ -13,13 +13,10 @@
 // occurrences costs its tiles no more than anyone else's.  Every sum has a fixed order (inside a
 // tile by sorted position, across tiles by tile index), no floating-point atomics anywhere.
 #include "segsort.cuh"
+#include "tile_reduce.cuh"
 
 namespace antdt {
 namespace {
-
-constexpr int kRedTile = 64;  // sorted occurrences per reduction tile (multiple of 32)
-constexpr int kRedThreads = 256;
-constexpr int kRedUnroll = 4;
 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -98,217 +95,6 @@ expand_bags_kernel(const int64_t* __restrict__ bag_offsets, int64_t n_bags, int6
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// Tile reduction.  A group of G lanes (one 16-byte vector of the row per lane and VPL step)
-// walks kRedTile = 64 consecutive sorted occurrences, summing gathered d_pooled rows; a run that
-// starts and ends inside the tile is written out (times 1/b_w), the pieces of runs that cross
-// the tile's edges go to head_part / tail_part for the fix-up pass.
-//
-// The kernel is issue-bound once a worker's d_pooled slice sits in L2, so the walk is built to
-// cost few instructions per occurrence: the tile's run ends are one 64-bit mask consumed with
-// constant shifts, the bag indices of G occurrences live in one register per lane and are
-// broadcast by shuffle, kRedUnroll row loads are in flight before the first add, and the
-// worker (for the 1/b_w scale) is only re-resolved when the walk crosses a worker boundary.
-// ---------------------------------------------------------------------------------------
-template <int G, int VPL>
-__global__ void __launch_bounds__(kRedThreads)
-seg_reduce_tiles_kernel(const uint32_t* __restrict__ sorted_occ, const uint32_t* __restrict__ head_bits,
-                        const int32_t* __restrict__ tile_first, const float* __restrict__ d_pooled,
-                        int dim, int64_t n, int64_t n_bags, const int64_t* __restrict__ occ_bounds,
-                        const float* __restrict__ worker_inv, int K, int64_t out_cap,
-                        float* __restrict__ uniq_grads, float* __restrict__ head_part,
-                        float* __restrict__ tail_part) {
-  extern __shared__ int64_t s_bounds[];  // [K+1]
-  for (int i = threadIdx.x; i <= K; i += blockDim.x) s_bounds[i] = occ_bounds[i];
-  __syncthreads();
-  const int lg = threadIdx.x & (G - 1);
-  const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
-  const int64_t o_begin = tile * kRedTile;
-  if (o_begin >= n) return;
-  const int nv = (int)min((int64_t)kRedTile, n - o_begin);  // occurrences in this tile
-  const unsigned gmask = group_mask<G>();
-  const int nvec = dim / 4;
-  constexpr int U = (G < kRedUnroll) ? G : kRedUnroll;
-
-  // run heads of positions o_begin .. o_begin+64; occurrence r closes its run iff r+1 is a head
-  const uint32_t* hw = head_bits + (o_begin >> 5);
-  const uint32_t h0 = __ldg(hw), h1 = __ldg(hw + 1), h2 = __ldg(hw + 2);
-  const uint64_t heads = (uint64_t)h0 | ((uint64_t)h1 << 32);
-  uint64_t ends = (heads >> 1) | ((uint64_t)(h2 & 1u) << 63);
-  const bool last_tile = o_begin + kRedTile >= n;
-  if (last_tile) ends = (ends & ((1ull << (nv - 1)) - 1ull)) | (1ull << (nv - 1));  // array end closes
-  const bool open_tail = !last_tile && !(h2 & 1u);  // the last run goes on in the next tile
-
-  int64_t u = tile_first[tile];
-  bool started = (h0 & 1u) != 0;
-  int w = interval_of(s_bounds, K + 1, o_begin);
-  if (w > K - 1) w = K - 1;
-  // tile-relative position at which the next worker starts (beyond the tile: never reached)
-  int next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
-  float inv = worker_inv[w];
-
-  float4 acc[VPL];
-#pragma unroll
-  for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-  const uint32_t row_stride = (uint32_t)dim;
-
-  for (int q = 0; q * G < nv; ++q) {
-    int my_bag = -1;
-    if (q * G + lg < nv) {
-      const uint32_t bg = __ldg(sorted_occ + o_begin + q * G + lg);
-      my_bag = ((int64_t)bg < n_bags) ? (int)bg : -1;  // -1: payload of a skipped (malformed) bag
-    }
-#pragma unroll
-    for (int j0 = 0; j0 < G; j0 += U) {
-      float4 v[U][VPL];
-#pragma unroll
-      for (int t = 0; t < U; ++t) {
-        const int bag = __shfl_sync(gmask, my_bag, j0 + t, G);
-        const float* rp = d_pooled + (size_t)((uint32_t)(bag < 0 ? 0 : bag)) * row_stride;
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-          const int vi = lg + k * G;
-          v[t][k] = (bag >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      }
-#pragma unroll
-      for (int t = 0; t < U; ++t) {
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-          acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
-          acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
-        }
-        if ((ends >> (j0 + t)) & 1ull) {  // this occurrence closes its run
-          float* dst;
-          float sc = 1.f;
-          if (started) {
-            const int rel = q * G + j0 + t;
-            if (rel >= next_w_rel) {  // crossed into a later worker's range
-              const int64_t o = o_begin + rel;
-              while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
-              next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
-              if (w == K - 1) next_w_rel = kRedTile + 1;
-              inv = worker_inv[w];
-            }
-            sc = inv;
-            dst = (u < out_cap) ? uniq_grads + (size_t)u * row_stride : nullptr;
-          } else {
-            dst = head_part + (size_t)tile * row_stride;
-          }
-          if (dst) {
-#pragma unroll
-            for (int k = 0; k < VPL; ++k) {
-              const int vi = lg + k * G;
-              if (vi < nvec)
-                reinterpret_cast<float4*>(dst)[vi] =
-                    make_float4(acc[k].x * sc, acc[k].y * sc, acc[k].z * sc, acc[k].w * sc);
-            }
-          }
-          ++u;
-          started = true;
-#pragma unroll
-          for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      }
-    }
-    ends = (G >= 64) ? 0ull : (ends >> (G & 63));
-  }
-  if (open_tail) {
-    float* dst = (started ? tail_part : head_part) + (size_t)tile * row_stride;
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-      const int vi = lg + k * G;
-      if (vi < nvec) reinterpret_cast<float4*>(dst)[vi] = acc[k];
-    }
-  }
-}
-
-// Fix-up: the tile in which a straddling run STARTS owns it.  total = its tail piece, then
-// the head pieces of the following tiles in order until the run ends.
-template <int G, int VPL>
-__global__ void __launch_bounds__(kRedThreads)
-seg_reduce_fixup_kernel(const uint32_t* __restrict__ head_bits, const int32_t* __restrict__ tile_first,
-                        int dim, int64_t n, const int64_t* __restrict__ occ_bounds,
-                        const float* __restrict__ worker_inv, int K, int64_t out_cap,
-                        float* __restrict__ uniq_grads, const float* __restrict__ head_part,
-                        const float* __restrict__ tail_part) {
-  const int lg = threadIdx.x & (G - 1);
-  const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
-  const int64_t o_begin = tile * kRedTile;
-  if (o_begin >= n) return;
-  const int64_t o_end = o_begin + kRedTile;
-  if (o_end >= n) return;  // the last tile's runs all end inside it
-  const int nvec = dim / 4;
-  uint32_t hb[kRedTile / 32 + 1];
-#pragma unroll
-  for (int i = 0; i <= kRedTile / 32; ++i) hb[i] = __ldg(head_bits + (o_begin >> 5) + i);
-  if (hb[kRedTile / 32] & 1u) return;  // next tile starts a new run: nothing straddles
-  int heads = 0;
-#pragma unroll
-  for (int i = 0; i < kRedTile / 32; ++i) heads += __popc(hb[i]);
-  if (heads == 0) return;  // the straddling run started earlier: its start tile owns it
-  const int64_t u = (int64_t)tile_first[tile] + heads - ((hb[0] & 1u) ? 1 : 0);
-  if (u >= out_cap) return;
-
-  float4 tot[VPL];
-#pragma unroll
-  for (int k = 0; k < VPL; ++k) {
-    const int vi = lg + k * G;
-    tot[k] = vi < nvec ? reinterpret_cast<const float4*>(tail_part + (size_t)tile * dim)[vi]
-                       : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  for (int64_t t2 = tile + 1;; ++t2) {
-    const int64_t b2 = t2 * kRedTile;
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-      const int vi = lg + k * G;
-      if (vi >= nvec) continue;
-      const float4 p = reinterpret_cast<const float4*>(head_part + (size_t)t2 * dim)[vi];
-      tot[k].x += p.x; tot[k].y += p.y; tot[k].z += p.z; tot[k].w += p.w;
-    }
-    if (b2 + kRedTile >= n) break;  // ran to the end of the array
-    bool ends = false;              // a head inside t2, or at the start of the tile after it
-#pragma unroll
-    for (int i = 0; i < kRedTile / 32; ++i) ends |= __ldg(head_bits + (b2 >> 5) + i) != 0u;
-    ends |= (__ldg(head_bits + (b2 >> 5) + kRedTile / 32) & 1u) != 0u;
-    if (ends) break;
-  }
-  // worker of the run = worker of any of its occurrences
-  int w = interval_of(occ_bounds, K + 1, o_end - 1);
-  if (w > K - 1) w = K - 1;
-  const float scale = worker_inv[w];
-  float* dst = uniq_grads + (size_t)u * dim;
-#pragma unroll
-  for (int k = 0; k < VPL; ++k) {
-    const int vi = lg + k * G;
-    if (vi >= nvec) continue;
-    float4 r = tot[k];
-    r.x *= scale; r.y *= scale; r.z *= scale; r.w *= scale;
-    reinterpret_cast<float4*>(dst)[vi] = r;
-  }
-}
-
-template <int G, int VPL>
-void launch_reduce(const BwdLayout& L, char* ws, const uint32_t* sorted_occ, const float* d_pooled,
-                   int dim, int64_t nnz, int64_t n_bags, int K, int64_t out_cap, float* uniq_grads,
-                   cudaStream_t s) {
-  const int64_t n_tiles = (nnz + kRedTile - 1) / kRedTile;
-  const int64_t tpb = kRedThreads / G;
-  const unsigned grid = (unsigned)((n_tiles + tpb - 1) / tpb);
-  const uint32_t* head_bits = (const uint32_t*)(ws + L.head_bits);
-  const int32_t* tile_first = (const int32_t*)(ws + L.tile_first);
-  const int64_t* occ_bounds = (const int64_t*)(ws + L.sort_ws + L.sort.seg_bounds);
-  const float* worker_b = (const float*)(ws + L.worker_b);
-  float* head_part = (float*)(ws + L.head_part);
-  float* tail_part = (float*)(ws + L.tail_part);
-  ANTDT_LAUNCH("seg_reduce_tiles", (seg_reduce_tiles_kernel<G, VPL>), grid, kRedThreads,
-               8 * ((size_t)K + 1), s, sorted_occ, head_bits, tile_first, d_pooled, dim, nnz,
-               n_bags, occ_bounds, worker_b, K, out_cap, uniq_grads, head_part, tail_part);
-  ANTDT_LAUNCH("seg_reduce_fixup", (seg_reduce_fixup_kernel<G, VPL>), grid, kRedThreads, 0, s,
-               head_bits, tile_first, dim, nnz, occ_bounds, worker_b, K, out_cap, uniq_grads,
-               head_part, tail_part);
-}
-
 }  // namespace
 }  // namespace antdt
 
@@ -374,19 +160,23 @@ extern "C" int32_t antdt_embbag_bwd_dedup(
                (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws,
                L.sort, dev_status, s);
   if (nnz > 0) {
-    const int nvec = dim / 4;
-#define RED_CASE(G, VPL)                                                                    \
-  launch_reduce<G, VPL>(L, w8, occ_out, d_pooled, dim, nnz, n_bags, K, out_cap, uniq_grads, s);
-    if (nvec <= 1) { RED_CASE(1, 1) }
-    else if (nvec <= 2) { RED_CASE(2, 1) }
-    else if (nvec <= 4) { RED_CASE(4, 1) }
-    else if (nvec <= 8) { RED_CASE(8, 1) }
-    else if (nvec <= 16) { RED_CASE(16, 1) }
-    else if (nvec <= 32) { RED_CASE(32, 1) }
-    else if (nvec <= 64) { RED_CASE(32, 2) }
-    else if (nvec <= 128) { RED_CASE(32, 4) }
-    else { RED_CASE(32, 8) }
-#undef RED_CASE
+    TileArgs t;
+    t.payload = occ_out;
+    t.head_bits = (const uint32_t*)(w8 + L.head_bits);
+    t.tile_first = (const int32_t*)(w8 + L.tile_first);
+    t.rows = d_pooled;
+    t.dim = dim;
+    t.n_host = nnz;
+    t.n_dev = nullptr;
+    t.payload_limit = n_bags;
+    t.bounds = (const int64_t*)(sort_ws + L.sort.seg_bounds);  // sanitised worker ranges
+    t.scales = d_worker_b;
+    t.K = K;
+    t.out_cap = out_cap;
+    t.out = uniq_grads;
+    t.head_part = (float*)(w8 + L.head_part);
+    t.tail_part = (float*)(w8 + L.tail_part);
+    launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
   }
   return cuda_ok();
 }

@@ -1,0 +1,280 @@
+// Tile-parallel segmented reduction of gathered rows, shared by the worker backward (sum of
+// d_pooled rows per (worker, row) run, scaled by 1/b_w) and the server aggregation (weighted sum
+// of the workers' gradient rows per row).
+//
+// The sorted array of payloads (row indices into `rows`) is cut into tiles of kRedTile = 64
+// consecutive entries whatever runs they belong to, so the work is balanced by entries, not by
+// runs: a run holding 20% of a field costs its tiles no more than anyone else's.  A group of G
+// lanes (one 16-byte vector of the row per lane and VPL step) walks one tile; a run that starts
+// and ends inside the tile is written out, the pieces of runs that cross the tile's edges go to
+// head_part / tail_part, and the fix-up pass lets the tile where such a run STARTS add its tail
+// piece and the following head pieces in tile order.  Every sum has a fixed order: no
+// floating-point atomics, bit-reproducible.
+//
+// The walk is issue-bound once the gathered rows sit in L2, so it is built to cost few
+// instructions per entry: the tile's run ends are one 64-bit mask consumed with constant
+// shifts, the payloads of G entries live in one register per lane and are broadcast by shuffle,
+// kRedUnroll row loads are in flight before the first add, and in the backward the worker (for
+// the 1/b_w scale) is only re-resolved when the walk crosses a worker boundary.
+#pragma once
+#include "common.cuh"
+
+namespace antdt {
+
+constexpr int kRedTile = 64;  // sorted entries per reduction tile (a power of two, multiple of 32)
+constexpr int kRedThreads = 256;
+constexpr int kRedUnroll = 4;
+
+struct TileArgs {
+  const uint32_t* payload;    // [n] sorted payloads: row index into `rows`
+  const uint32_t* head_bits;  // bit i set iff entry i starts a run
+  const int32_t* tile_first;  // run index of entry t*kRedTile
+  const float* rows;          // gathered matrix [payload_limit, dim]
+  int dim;
+  int64_t n_host;             // entries (upper bound when n_dev is given)
+  const int64_t* n_dev;       // device-side entry count or nullptr
+  int64_t payload_limit;      // payloads >= this are skipped (never dereferenced)
+  const int64_t* bounds;      // backward: entry range of every worker [K+1];
+                              // aggregation: payload range of every worker [K+1]
+  const float* scales;        // backward: 1/b_w [K]; aggregation: weight w_i [K]
+  int K;
+  int64_t out_cap;
+  float* out;                 // [out_cap, dim]
+  float* head_part;           // [n_tiles, dim]
+  float* tail_part;           // [n_tiles, dim]
+};
+
+// The hot pointers are separate __restrict__ parameters (not read through the struct) so that
+// the compiler may move row loads across the run-end stores.
+template <int G, int VPL, bool AGG>
+__global__ void __launch_bounds__(kRedThreads, (VPL == 1 ? 5 : 1))
+tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
+                   const uint32_t* __restrict__ head_bits, const int32_t* __restrict__ tile_first,
+                   const float* __restrict__ rows, float* __restrict__ out,
+                   float* __restrict__ head_part, float* __restrict__ tail_part) {
+  extern __shared__ int64_t s_bounds[];  // [K+1], then K floats (aggregation)
+  float* s_w = reinterpret_cast<float*>(s_bounds + (a.K + 1));
+  const int K = a.K;
+  for (int i = threadIdx.x; i <= K; i += blockDim.x) s_bounds[i] = a.bounds[i];
+  if (AGG)
+    for (int i = threadIdx.x; i < K; i += blockDim.x) s_w[i] = a.scales[i];
+  __syncthreads();
+  const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
+  const int lg = threadIdx.x & (G - 1);
+  const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
+  const int64_t o_begin = tile * kRedTile;
+  if (o_begin >= n) return;
+  const int nv = (int)min((int64_t)kRedTile, n - o_begin);  // entries in this tile
+  const unsigned gmask = group_mask<G>();
+  const int dim = a.dim;
+  const int nvec = dim / 4;
+  constexpr int U = (G < kRedUnroll) ? G : kRedUnroll;
+
+  // run heads of positions o_begin .. o_begin+64; entry r closes its run iff r+1 is a head
+  const uint32_t* hw = head_bits + (o_begin >> 5);
+  const uint32_t h0 = __ldg(hw), h1 = __ldg(hw + 1), h2 = __ldg(hw + 2);
+  const uint64_t heads = (uint64_t)h0 | ((uint64_t)h1 << 32);
+  uint64_t ends = (heads >> 1) | ((uint64_t)(h2 & 1u) << 63);
+  const bool last_tile = o_begin + kRedTile >= n;
+  if (last_tile) ends = (ends & ((1ull << (nv - 1)) - 1ull)) | (1ull << (nv - 1));  // array end closes
+  const bool open_tail = !last_tile && !(h2 & 1u);  // the last run goes on in the next tile
+
+  int64_t u = tile_first[tile];
+  bool started = (h0 & 1u) != 0;
+  int w = 0, next_w_rel = kRedTile + 1;
+  float inv = 1.f;
+  if (!AGG) {
+    w = interval_of(s_bounds, K + 1, o_begin);
+    if (w > K - 1) w = K - 1;
+    // tile-relative position at which the next worker starts (beyond the tile: never reached)
+    next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
+    inv = a.scales[w];
+  }
+
+  float4 acc[VPL];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  const uint32_t row_stride = (uint32_t)dim;
+
+  for (int q = 0; q * G < nv; ++q) {
+    int my_row = -1;
+    float my_wt = 0.f;
+    if (q * G + lg < nv) {
+      const uint32_t p = __ldg(payload + o_begin + q * G + lg);
+      my_row = ((int64_t)p < a.payload_limit) ? (int)p : -1;  // -1: skipped, contributes nothing
+      if (AGG && my_row >= 0) {
+        int wl = interval_of(s_bounds, K + 1, (int64_t)p);
+        my_wt = s_w[wl > K - 1 ? K - 1 : wl];
+      }
+    }
+#pragma unroll
+    for (int j0 = 0; j0 < G; j0 += U) {
+      float4 v[U][VPL];
+      float wt[U];
+#pragma unroll
+      for (int t = 0; t < U; ++t) {
+        const int row = __shfl_sync(gmask, my_row, j0 + t, G);
+        wt[t] = AGG ? __shfl_sync(gmask, my_wt, j0 + t, G) : 1.f;
+        const float* rp = rows + (size_t)((uint32_t)(row < 0 ? 0 : row)) * row_stride;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          const int vi = lg + k * G;
+          v[t][k] = (row >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < U; ++t) {
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          if (AGG) {
+            acc[k].x = fmaf(wt[t], v[t][k].x, acc[k].x); acc[k].y = fmaf(wt[t], v[t][k].y, acc[k].y);
+            acc[k].z = fmaf(wt[t], v[t][k].z, acc[k].z); acc[k].w = fmaf(wt[t], v[t][k].w, acc[k].w);
+          } else {
+            acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
+            acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
+          }
+        }
+        if ((ends >> (j0 + t)) & 1ull) {  // this entry closes its run
+          float* dst;
+          float sc = 1.f;
+          if (started) {
+            if (!AGG) {
+              const int rel = q * G + j0 + t;
+              if (rel >= next_w_rel) {  // crossed into a later worker's range
+                const int64_t o = o_begin + rel;
+                while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
+                next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
+                if (w == K - 1) next_w_rel = kRedTile + 1;
+                inv = a.scales[w];
+              }
+              sc = inv;
+            }
+            dst = (u < a.out_cap) ? out + (size_t)u * row_stride : nullptr;
+          } else {
+            dst = head_part + (size_t)tile * row_stride;
+          }
+          if (dst) {
+#pragma unroll
+            for (int k = 0; k < VPL; ++k) {
+              const int vi = lg + k * G;
+              if (vi < nvec)
+                reinterpret_cast<float4*>(dst)[vi] =
+                    AGG ? acc[k]
+                        : make_float4(acc[k].x * sc, acc[k].y * sc, acc[k].z * sc, acc[k].w * sc);
+            }
+          }
+          ++u;
+          started = true;
+#pragma unroll
+          for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    }
+    ends = (G >= 64) ? 0ull : (ends >> (G & 63));
+  }
+  if (open_tail) {
+    float* dst = (started ? tail_part : head_part) + (size_t)tile * row_stride;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+      const int vi = lg + k * G;
+      if (vi < nvec) reinterpret_cast<float4*>(dst)[vi] = acc[k];
+    }
+  }
+}
+
+// Fix-up: the tile in which a straddling run STARTS owns it.  total = its tail piece, then
+// the head pieces of the following tiles in order until the run ends.
+template <int G, int VPL, bool AGG>
+__global__ void __launch_bounds__(kRedThreads)
+tile_fixup_kernel(const TileArgs a) {
+  const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
+  const int lg = threadIdx.x & (G - 1);
+  const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
+  const int64_t o_begin = tile * kRedTile;
+  if (o_begin >= n) return;
+  const int64_t o_end = o_begin + kRedTile;
+  if (o_end >= n) return;  // the last tile's runs all end inside it
+  const int dim = a.dim;
+  const int nvec = dim / 4;
+  uint32_t hb[kRedTile / 32 + 1];
+#pragma unroll
+  for (int i = 0; i <= kRedTile / 32; ++i) hb[i] = __ldg(a.head_bits + (o_begin >> 5) + i);
+  if (hb[kRedTile / 32] & 1u) return;  // next tile starts a new run: nothing straddles
+  int heads = 0;
+#pragma unroll
+  for (int i = 0; i < kRedTile / 32; ++i) heads += __popc(hb[i]);
+  if (heads == 0) return;  // the straddling run started earlier: its start tile owns it
+  const int64_t u = (int64_t)a.tile_first[tile] + heads - ((hb[0] & 1u) ? 1 : 0);
+  if (u >= a.out_cap) return;
+
+  float4 tot[VPL];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int vi = lg + k * G;
+    tot[k] = vi < nvec ? reinterpret_cast<const float4*>(a.tail_part + (size_t)tile * dim)[vi]
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int64_t t2 = tile + 1;; ++t2) {
+    const int64_t b2 = t2 * kRedTile;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+      const int vi = lg + k * G;
+      if (vi >= nvec) continue;
+      const float4 p = reinterpret_cast<const float4*>(a.head_part + (size_t)t2 * dim)[vi];
+      tot[k].x += p.x; tot[k].y += p.y; tot[k].z += p.z; tot[k].w += p.w;
+    }
+    if (b2 + kRedTile >= n) break;  // ran to the end of the array
+    bool ends = false;              // a head inside t2, or at the start of the tile after it
+#pragma unroll
+    for (int i = 0; i < kRedTile / 32; ++i) ends |= __ldg(a.head_bits + (b2 >> 5) + i) != 0u;
+    ends |= (__ldg(a.head_bits + (b2 >> 5) + kRedTile / 32) & 1u) != 0u;
+    if (ends) break;
+  }
+  float scale = 1.f;
+  if (!AGG) {  // worker of the run = worker of any of its entries
+    int w = interval_of(a.bounds, a.K + 1, o_end - 1);
+    if (w > a.K - 1) w = a.K - 1;
+    scale = a.scales[w];
+  }
+  float* dst = a.out + (size_t)u * dim;
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int vi = lg + k * G;
+    if (vi >= nvec) continue;
+    float4 r = tot[k];
+    if (!AGG) { r.x *= scale; r.y *= scale; r.z *= scale; r.w *= scale; }
+    reinterpret_cast<float4*>(dst)[vi] = r;
+  }
+}
+
+template <int G, int VPL, bool AGG>
+void launch_tile_reduce_gv(const TileArgs& a, const char* name_tiles, const char* name_fixup,
+                           cudaStream_t s) {
+  const int64_t n_tiles = (a.n_host + kRedTile - 1) / kRedTile;
+  const int64_t tpb = kRedThreads / G;
+  const unsigned grid = (unsigned)((n_tiles + tpb - 1) / tpb);
+  if (grid == 0) return;
+  const size_t smem = 8 * ((size_t)a.K + 1) + (AGG ? 4 * (size_t)a.K : 0);
+  ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, AGG>), grid, kRedThreads, smem, s, a, a.payload,
+               a.head_bits, a.tile_first, a.rows, a.out, a.head_part, a.tail_part);
+  ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, AGG>), grid, kRedThreads, 0, s, a);
+}
+
+template <bool AGG>
+void launch_tile_reduce(const TileArgs& a, const char* name_tiles, const char* name_fixup,
+                        cudaStream_t s) {
+  const int nvec = a.dim / 4;
+#define TILE_CASE(G, VPL) launch_tile_reduce_gv<G, VPL, AGG>(a, name_tiles, name_fixup, s)
+  if (nvec <= 1) TILE_CASE(1, 1);
+  else if (nvec <= 2) TILE_CASE(2, 1);
+  else if (nvec <= 4) TILE_CASE(4, 1);
+  else if (nvec <= 8) TILE_CASE(8, 1);
+  else if (nvec <= 16) TILE_CASE(16, 1);
+  else if (nvec <= 32) TILE_CASE(32, 1);
+  else if (nvec <= 64) TILE_CASE(32, 2);
+  else if (nvec <= 128) TILE_CASE(32, 4);
+  else TILE_CASE(32, 8);
+#undef TILE_CASE
+}
+
+}  // namespace antdt

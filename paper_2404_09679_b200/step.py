@@ -45,7 +45,7 @@ class StepBuffers:
         self.status = torch.zeros(1, dtype=i32, device=dev)
         self.dense_out = torch.empty(dense_n, dtype=f32, device=dev) if dense_n else None
         ws_bytes = max(B.antdt_embbag_bwd_dedup_workspace_bytes(max_nnz, max_bags, dim, n_workers),
-                       B.antdt_weighted_aggregate_workspace_bytes(self.uniq_cap, n_workers))
+                       B.antdt_weighted_aggregate_workspace_bytes(self.uniq_cap, dim, n_workers))
         self.ws = torch.empty((ws_bytes + 255) // 256 * 256, dtype=torch.uint8, device=dev)
 
 

@@ -101,7 +101,7 @@ def gpu_aggregate(uniq_ids, wuo, uniq_grads, bsz, n_rows, dense=None, out_cap=No
     agg_ids = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
     agg = torch.full((cap, D), float("nan"), device="cuda")
     n_agg = torch.full((1,), -1, dtype=torch.int64, device="cuda")
-    ws = torch.empty(B.antdt_weighted_aggregate_workspace_bytes(ug.shape[0], K), dtype=torch.uint8,
+    ws = torch.empty(B.antdt_weighted_aggregate_workspace_bytes(ug.shape[0], D, K), dtype=torch.uint8,
                      device="cuda")
     st = new_status()
     dg = dout = None

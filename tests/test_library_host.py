@@ -65,8 +65,8 @@ def test_device_calls_reject_bad_arguments_before_any_launch():
     assert L.antdt_sparse_opt_update(one, B.F32, 10, 8, one, one, one, 4, B.OPT_ADAGRAD, 0.1, 1e-8, 0.9,
                                      0.999, 0, one, None, None, None) == B.ERR_INVALID_ARG  # step 0
     assert B.antdt_launch_count() == n0
-    assert B.antdt_weighted_aggregate_workspace_bytes(100, 4) > 0
-    assert B.antdt_weighted_aggregate_workspace_bytes(100, 2000) == 0
+    assert B.antdt_weighted_aggregate_workspace_bytes(100, 16, 4) > 0
+    assert B.antdt_weighted_aggregate_workspace_bytes(100, 16, 2000) == 0
 
 
 # ---- planner: library vs checker, bit for bit ---------------------------------------------
