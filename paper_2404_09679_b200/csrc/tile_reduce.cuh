@@ -47,7 +47,7 @@ struct TileArgs {
 // The hot pointers are separate __restrict__ parameters (not read through the struct) so that
 // the compiler may move row loads across the run-end stores.
 template <int G, int VPL, bool AGG>
-__global__ void __launch_bounds__(kRedThreads, (VPL == 1 ? 5 : 1))
+__global__ void __launch_bounds__(kRedThreads, (VPL == 1 ? 6 : 1))
 tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
                    const uint32_t* __restrict__ head_bits, const int32_t* __restrict__ tile_first,
                    const float* __restrict__ rows, float* __restrict__ out,
