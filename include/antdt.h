@@ -265,9 +265,11 @@ int32_t antdt_sparse_opt_update(void* table, int32_t dtype, int64_t n_rows, int3
 
 /* One whole step from HOST buffers: copies the step's inputs to the caller's device staging
  * buffers, runs fwd, bwd_dedup, aggregate and update in order on `stream`, and copies the
- * results (pooled, dense_out, n_agg, status) back; all asynchronous on `stream`, the caller
- * synchronises.  Host buffers should be page-locked for the copies to overlap.  Every
- * pointer of the descriptor is described beside its field. */
+ * results (pooled, dense_out, n_agg, status) back.  The copies run on two internal side
+ * streams (created on the first call on a device) so that they overlap the kernels; `stream`
+ * waits for all of them before the call's work on it ends, so synchronising `stream` is enough.
+ * Host buffers should be page-locked for the copies to overlap.  Every pointer of the
+ * descriptor is described beside its field. */
 typedef struct {
   /* model state, device resident */
   void* table; int32_t dtype; int64_t n_rows; int32_t dim;

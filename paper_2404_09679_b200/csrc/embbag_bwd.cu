@@ -105,13 +105,16 @@ extern "C" size_t antdt_embbag_bwd_dedup_workspace_bytes(int64_t nnz, int64_t n_
   return antdt::bwd_layout(nnz, dim, n_workers).bytes;
 }
 
-extern "C" int32_t antdt_embbag_bwd_dedup(
+namespace antdt {
+// The entry point's body.  d_pooled is first read by the tile reduction; a caller that is still
+// copying it in on another stream passes the event that marks its arrival (the sort and the
+// run detection, which only need the ids, then overlap the copy).
+int32_t bwd_dedup_impl(
     const int32_t* row_ids, int64_t nnz, const int64_t* bag_offsets, int64_t n_bags,
     int32_t bags_per_sample, const float* d_pooled, int32_t dim, int64_t n_rows, int32_t n_workers,
     const int64_t* worker_sample_offsets, int32_t* uniq_ids, int64_t* worker_uniq_offsets,
     int64_t* seg_offsets, int32_t* sorted_occ, float* uniq_grads, int64_t out_cap, void* ws,
-    size_t ws_bytes, int32_t* dev_status, void* stream) {
-  using namespace antdt;
+    size_t ws_bytes, int32_t* dev_status, void* stream, cudaEvent_t d_pooled_ready) {
   const int K = n_workers;
   if (nnz < 0 || n_bags < 0 || nnz >= (1ll << 31) || n_bags >= (1ll << 31) || n_rows < 1 ||
       n_rows >= (1ll << 31) || dim < 4 || dim > 1024 || dim % 4 || K < 1 || K > kMaxSegments ||
@@ -159,6 +162,8 @@ extern "C" int32_t antdt_embbag_bwd_dedup(
   segsort_runs(keys_a, nnz, uniq_ids, seg_offsets, worker_uniq_offsets, nullptr, out_cap,
                (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws,
                L.sort, dev_status, s);
+  if (d_pooled_ready && cudaStreamWaitEvent(s, d_pooled_ready, 0) != cudaSuccess)
+    return ANTDT_ERR_CUDA;
   if (nnz > 0) {
     TileArgs t;
     t.payload = occ_out;
@@ -179,4 +184,17 @@ extern "C" int32_t antdt_embbag_bwd_dedup(
     launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
   }
   return cuda_ok();
+}
+}  // namespace antdt
+
+extern "C" int32_t antdt_embbag_bwd_dedup(
+    const int32_t* row_ids, int64_t nnz, const int64_t* bag_offsets, int64_t n_bags,
+    int32_t bags_per_sample, const float* d_pooled, int32_t dim, int64_t n_rows, int32_t n_workers,
+    const int64_t* worker_sample_offsets, int32_t* uniq_ids, int64_t* worker_uniq_offsets,
+    int64_t* seg_offsets, int32_t* sorted_occ, float* uniq_grads, int64_t out_cap, void* ws,
+    size_t ws_bytes, int32_t* dev_status, void* stream) {
+  return antdt::bwd_dedup_impl(row_ids, nnz, bag_offsets, n_bags, bags_per_sample, d_pooled, dim,
+                               n_rows, n_workers, worker_sample_offsets, uniq_ids,
+                               worker_uniq_offsets, seg_offsets, sorted_occ, uniq_grads, out_cap, ws,
+                               ws_bytes, dev_status, stream, nullptr);
 }
