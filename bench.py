@@ -141,6 +141,12 @@ def plan_all(w, n_steps):
     return plans
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
+# full-size default workload summarised in profiles/; a kernel that has changed since is set to None.
+NCU_TRAFFIC = {4: {"seg_reduce_tiles": 12.95e9, "agg_reduce": 6.80e9, "sparse_adagrad": 9.42e9,
+                   "embbag_fwd": 4.04e9, "radix_scatter": (2.96e9 + 2.39e9 + 2.11e9) / 3}}
+
+
 def scaled_workload(w, scale):
     if scale == 1.0:
         return w
@@ -156,6 +162,10 @@ def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
     D, ew = w.D, (2 if w.table_dtype == "bf16" else 4)
     S = 2 if w.opt == "adam" else 1
     return {
+        "radix_hist": 4 * nnz, "radix_scatter": 16 * nnz, "runs_count": 4 * nnz,
+        "runs_emit": 4 * nnz + nnz // 8 + 12 * sum_u,
+        "agg_radix_hist": 4 * sum_u, "agg_radix_scatter": 16 * sum_u, "agg_runs_count": 4 * sum_u,
+        "agg_runs_emit": 4 * sum_u + sum_u // 8 + 12 * u,
         "embbag_fwd": 4 * nnz + 8 * (n_bags + 1) + nnz * D * ew + n_bags * D * 4,
         "expand_bags": 8 * (n_bags + 1) + 4 * nnz,
         "seg_reduce_tiles": 4 * nnz + nnz // 8 + nnz * D * 4 + sum_u * D * 4,
@@ -169,7 +179,9 @@ def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
 def step_bytes(w, nnz, n_bags, sum_u, u, passes_bwd, passes_agg):
     b = algorithmic_bytes(w, nnz, n_bags, sum_u, u)
     upd = b["sparse_adam"] if w.opt == "adam" else b["sparse_adagrad"]
-    sort = passes_bwd * 20 * nnz + passes_agg * 20 * sum_u + 8 * nnz + 8 * sum_u
+    sort = (passes_bwd * (b["radix_hist"] + b["radix_scatter"]) + b["runs_count"] + b["runs_emit"] +
+            passes_agg * (b["agg_radix_hist"] + b["agg_radix_scatter"]) + b["agg_runs_count"] +
+            b["agg_runs_emit"])
     return (b["embbag_fwd"] + b["expand_bags"] + b["seg_reduce_tiles"] + b["agg_reduce"] + upd +
             (b["dense_wsum"] if w.dense_n else 0) + sort)
 
@@ -242,7 +254,7 @@ class OracleSample:
 
 # samples per worker in the bounded sample: about 15 s of checker time for the baseline leg of
 # our arm, about 5 s per step for the reference arm (which runs warmup + steps of them)
-CPU_SAMPLE_PER_WORKER = {1: 1 << 30, 2: 1 << 30, 3: 768, 4: 768, 5: 4096}
+CPU_SAMPLE_PER_WORKER = {1: 1 << 30, 2: 1 << 30, 3: 1536, 4: 2048, 5: 8192}
 REF_SAMPLE_PER_WORKER = {1: 1 << 30, 2: 1 << 30, 3: 256, 4: 256, 5: 1536}
 
 
@@ -396,6 +408,10 @@ def run_ours(args):
     if top in alg:
         roof["achieved"] = round(alg[top] / (top_ms / top_n * 1e-3) / 1e9, 1)
         roof["frac"] = round(roof["achieved"] / peak_gbs, 4)
+    if args.scale == 1.0 and world == 1:
+        roof["traffic"] = NCU_TRAFFIC.get(cfg, {}).get(top)
+        if roof["traffic"]:
+            roof["dram_GBps_from_traffic"] = round(roof["traffic"] / (top_ms / top_n * 1e-3) / 1e9, 1)
     rowbits = max(1, (w.V - 1).bit_length())
     passes = -(-rowbits // 9)
     sb = step_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen, passes, passes)

@@ -155,10 +155,10 @@ extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const a
     segsort_setup(bounds, 1, in_cap, sort_ws, L.sort, s);
     segsort_run(reinterpret_cast<const uint32_t*>(sp->uniq_ids), nullptr, keys_a,
                 (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b), (uint32_t*)(w8 + L.vals_t),
-                bits_for(sp->n_rows), 0, sort_ws, L.sort, dev_status, s);
+                bits_for(sp->n_rows), 0, sort_ws, L.sort, dev_status, s, true);
     segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
                  sp->out_cap < in_cap ? sp->out_cap : in_cap, (uint32_t*)(w8 + L.head_bits),
-                 (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s);
+                 (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s, true);
     if (in_cap > 0) {
       TileArgs t;
       t.payload = (const uint32_t*)(w8 + L.src);

@@ -523,7 +523,7 @@ void segsort_setup(const int64_t* seg_bounds_dev, int S, int64_t n_cap, char* ws
 void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* keys_out,
                  uint32_t* vals_out, uint32_t* keys_tmp, uint32_t* vals_tmp, int key_bits,
                  int64_t check_rows, char* ws, const SortLayout& L, int32_t* status,
-                 cudaStream_t s) {
+                 cudaStream_t s, bool agg) {
   const SortDesc* desc = (const SortDesc*)(ws + L.desc);
   const int64_t* seg_bounds = (const int64_t*)(ws + L.seg_bounds);
   const int32_t* seg_first = (const int32_t*)(ws + L.seg_first);
@@ -553,11 +553,11 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
     const bool to_out = ((P - 1 - p) % 2) == 0;
     uint32_t* kout = to_out ? keys_out : keys_tmp;
     uint32_t* vout = to_out ? vals_out : vals_tmp;
-    ANTDT_LAUNCH("radix_hist", radix_hist_kernel, L.max_chunks, kSortThreads, 0, s, kin, shift,
+    ANTDT_LAUNCH(agg ? "agg_radix_hist" : "radix_hist", radix_hist_kernel, L.max_chunks, kSortThreads, 0, s, kin, shift,
                  mask, desc, chunk_begin, chunk_end, hist, p == 0 ? check_rows : (int64_t)0, status);
-    ANTDT_LAUNCH("radix_scan", radix_scan_kernel, S, kSortMaxBins, 0, s, desc, seg_first, hist,
+    ANTDT_LAUNCH(agg ? "agg_radix_scan" : "radix_scan", radix_scan_kernel, S, kSortMaxBins, 0, s, desc, seg_first, hist,
                  bin_base);
-    ANTDT_LAUNCH("radix_scatter", radix_scatter_kernel, L.max_chunks, kScatThreads, kScatSmem, s, kin, vin,
+    ANTDT_LAUNCH(agg ? "agg_radix_scatter" : "radix_scatter", radix_scatter_kernel, L.max_chunks, kScatThreads, kScatSmem, s, kin, vin,
                  kout, vout, shift, mask, desc, chunk_seg, seg_bounds, chunk_begin, chunk_end, hist,
                  bin_base);
     kin = kout;
@@ -569,7 +569,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
 void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys,
                   int64_t* run_start, int64_t* seg_runs, int64_t* n_runs_out, int64_t out_cap,
                   uint32_t* head_bits, int32_t* tile_first, int tile, char* ws,
-                  const SortLayout& L, int32_t* status, cudaStream_t s) {
+                  const SortLayout& L, int32_t* status, cudaStream_t s, bool agg) {
   const SortDesc* desc = (const SortDesc*)(ws + L.desc);
   const int64_t* seg_bounds = (const int64_t*)(ws + L.seg_bounds);
   const int32_t* seg_first = (const int32_t*)(ws + L.seg_first);
@@ -580,11 +580,11 @@ void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys
   if (head_bits) cudaMemsetAsync(head_bits, 0, head_bits_words(n_cap) * 4, s);
   int tile_shift = 0;
   while ((1 << tile_shift) < tile) ++tile_shift;  // tile is a power of two
-  ANTDT_LAUNCH("runs_count", runs_count_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys,
+  ANTDT_LAUNCH(agg ? "agg_runs_count" : "runs_count", runs_count_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys,
                desc, chunk_seg, seg_bounds, chunk_begin, chunk_end, chunk_runs);
-  ANTDT_LAUNCH("runs_scan", runs_scan_kernel, 1, 1024, 0, s, desc, seg_first, chunk_runs, seg_runs,
+  ANTDT_LAUNCH(agg ? "agg_runs_scan" : "runs_scan", runs_scan_kernel, 1, 1024, 0, s, desc, seg_first, chunk_runs, seg_runs,
                n_runs_out, run_start, out_cap, status);
-  ANTDT_LAUNCH("runs_emit", runs_emit_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys, desc,
+  ANTDT_LAUNCH(agg ? "agg_runs_emit" : "runs_emit", runs_emit_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys, desc,
                chunk_seg, seg_bounds, chunk_begin, chunk_end, chunk_runs, uniq_keys, run_start,
                out_cap, head_bits, tile_first, tile_shift);
 }

@@ -67,10 +67,11 @@ void segsort_setup(const int64_t* seg_bounds_dev, int n_segments, int64_t n_cap,
 // Sorts by the low key_bits bits.  keys_in is read only; the sorted pairs land in
 // keys_out/vals_out; keys_tmp/vals_tmp are scratch of the same size.  vals_in == nullptr means
 // "value = element index".  check_rows > 0: keys >= check_rows raise ID_OUT_OF_RANGE.
+// agg only selects the names under which the launches are accounted.
 void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* keys_out,
                  uint32_t* vals_out, uint32_t* keys_tmp, uint32_t* vals_tmp, int key_bits,
                  int64_t check_rows, char* ws, const SortLayout& L, int32_t* status,
-                 cudaStream_t s);
+                 cudaStream_t s, bool agg = false);
 
 // Runs of equal keys inside the segments of a sorted array.
 //   uniq_keys  [out_cap]    key of each run, in array order
@@ -83,6 +84,6 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
 void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys,
                   int64_t* run_start, int64_t* seg_runs, int64_t* n_runs_out, int64_t out_cap,
                   uint32_t* head_bits, int32_t* tile_first, int tile, char* ws,
-                  const SortLayout& L, int32_t* status, cudaStream_t s);
+                  const SortLayout& L, int32_t* status, cudaStream_t s, bool agg = false);
 
 }  // namespace antdt
