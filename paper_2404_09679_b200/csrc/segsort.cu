@@ -245,10 +245,9 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
   extern __shared__ __align__(16) unsigned char scat_smem[];
   uint32_t* gbase = reinterpret_cast<uint32_t*>(scat_smem);  // next global slot of every bin
   uint32_t* bin_start = gbase + kSortMaxBins;                // first slot of every bin in the tile
-  uint32_t* bin_cnt = bin_start + kSortMaxBins;
-  uint32_t* skeys = bin_cnt + kSortMaxBins;
-  uint32_t* svals = skeys + kSortTile;
-  uint32_t* warp_tot = svals + kSortTile;                    // [16]
+  uint32_t* bin_cnt = bin_start + kSortMaxBins;              // gbase - bin_start of the current tile
+  uint2* spairs = reinterpret_cast<uint2*>(bin_cnt + kSortMaxBins);  // (key, value), 8-byte aligned
+  uint32_t* warp_tot = reinterpret_cast<uint32_t*>(spairs + kSortTile);  // [16]
   unsigned short* wh = reinterpret_cast<unsigned short*>(warp_tot + 16);  // [16][512]
 
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -302,7 +301,6 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
         wh[ww * kSortMaxBins + tid] = (unsigned short)sum;
         sum += t;
       }
-      bin_cnt[tid] = sum;
       // exclusive scan over the 512 bins
       uint32_t incl = sum;
 #pragma unroll
@@ -315,7 +313,10 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
       uint32_t wp = 0;
 #pragma unroll
       for (int ww = 0; ww < kScatWarps; ++ww) wp += (ww < w) ? warp_tot[ww] : 0u;
-      bin_start[tid] = incl - sum + wp;
+      const uint32_t bs = incl - sum + wp;
+      bin_start[tid] = bs;
+      bin_cnt[tid] = gbase[tid] - bs;  // global slot of tile slot j in this bin = j + this
+      gbase[tid] += sum;               // for the next tile (only this thread touches its bin)
     }
     __syncthreads();  // (D)
 
@@ -324,8 +325,7 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
       if (wbase + i * 32 < tile_n) {
         const uint32_t d = (k[i] >> shift) & mask;
         const uint32_t p = bin_start[d] + my_wh[d] + rank[i];
-        skeys[p] = k[i];
-        svals[p] = v[i];
+        spairs[p] = make_uint2(k[i], v[i]);
       }
     }
     __syncthreads();  // (E)
@@ -334,15 +334,13 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
     for (int i = 0; i < kScatItems; ++i) {
       const int j = tid + i * kScatThreads;
       if (j < tile_n) {
-        const uint32_t kk = skeys[j];
-        const uint32_t d = (kk >> shift) & mask;
-        const uint32_t g = gbase[d] + ((uint32_t)j - bin_start[d]);
-        keys_out[g] = kk;
-        vals_out[g] = svals[j];
+        const uint2 kv = spairs[j];
+        const uint32_t g = bin_cnt[(kv.x >> shift) & mask] + (uint32_t)j;
+        keys_out[g] = kv.x;
+        vals_out[g] = kv.y;
       }
     }
-    __syncthreads();  // (F)
-    gbase[tid] += bin_cnt[tid];
+    // the next tile's barrier (A) orders these reads before the next (D) rewrites bin_cnt
   }
 }
 
@@ -533,8 +531,11 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
   uint32_t* hist = (uint32_t*)(ws + L.hist);
   uint32_t* bin_base = (uint32_t*)(ws + L.bin_base);
   const int P = sort_passes(key_bits);
-  static bool carveout_set = false;
-  if (!carveout_set) {  // 4 CTAs x 46 KB of shared memory per SM need the large carve-out
+  static bool attr_set[64] = {};
+  int dev_id = 0;
+  cudaGetDevice(&dev_id);
+  bool& carveout_set = attr_set[dev_id & 63];
+  if (!carveout_set) {  // per device: opt in to 55 KB of dynamic shared memory, 3 CTAs per SM
     cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)kScatSmem);
     cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,

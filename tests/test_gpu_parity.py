@@ -285,3 +285,41 @@ def test_update_textbook_cases_and_flags():
                                     np.zeros((4, 8), np.float32))
     assert code == B.ERR_ID_OUT_OF_RANGE
     assert np.all(gw[[0, 3]] == 1.0) and np.all(gw[[1, 2]] == 0.5) and np.all(acc[[1, 2]] == 1.0)
+
+
+# ---- limits of the worker count, and the parts of the aggregate on their own ------------------
+def test_a_thousand_workers():
+    rng = np.random.default_rng(41)
+    V, D, K, F, S = 5000, 16, 1000, 2, 3000
+    ids, off = random_bags(rng, S * F, V, 6, zipf=1.2)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    wso = _wso(rng, K, S, empties=True)
+    got, want = _check_bwd(ids, off, F, dY, V, wso)
+    bsz = np.maximum(np.diff(wso), 0)
+    aid, agg, na, _, code = G.gpu_aggregate(got["uniq_ids"], got["worker_uniq_offsets"],
+                                            got["uniq_grads"], bsz, V)
+    assert code == 0
+    want_ids, want_agg = oracle.aggregate_sparse(want["uniq_ids"], want["worker_uniq_offsets"],
+                                                 want["uniq_grads"], bsz)
+    assert np.array_equal(aid, want_ids)
+    G.close(agg, want_agg, rtol=3e-5, atol=2e-6)
+
+
+def test_dense_part_alone_and_sparse_part_alone():
+    rng = np.random.default_rng(42)
+    K, n = 6, 40_000
+    g = rng.normal(size=(K, n)).astype(np.float32)
+    bsz = rng.integers(1, 100, size=K)
+    dg, out = G.dev(g), torch.full((n,), float("nan"), device="cuda")
+    ws = torch.empty(B.antdt_weighted_aggregate_workspace_bytes(0, 0, K), dtype=torch.uint8, device="cuda")
+    st = G.new_status()
+    B.antdt_weighted_aggregate([int(b) for b in bsz], ws, dense_grads=dg, dense_out=out, dev_status=st)
+    assert B.antdt_read_status(st) == 0
+    G.close(out.cpu().numpy(), oracle.aggregate_dense(g, bsz))
+    # a strided view: worker vectors 2n apart
+    wide = torch.zeros(K, 2 * n, device="cuda")
+    wide[:, :n] = dg
+    out.fill_(float("nan"))
+    B.antdt_weighted_aggregate([int(b) for b in bsz], ws, dense_grads=wide[:, :n], dense_out=out,
+                               dev_status=st)
+    G.close(out.cpu().numpy(), oracle.aggregate_dense(g, bsz))
