@@ -59,7 +59,8 @@ enum {
   ANTDT_ERR_TIMEOUT = 6,             /* a bounded device-side wait ran out                */
   ANTDT_ERR_EXHAUSTED = 7,           /* the shard queue is empty: the epoch is over       */
   ANTDT_ERR_STATE = 8,               /* call not valid in the handle's current state      */
-  ANTDT_ERR_BAD_OFFSETS = 9          /* device saw bag offsets that do not ascend / fit   */
+  ANTDT_ERR_BAD_OFFSETS = 9,         /* device saw bag offsets that do not ascend / fit   */
+  ANTDT_ERR_INFEASIBLE = 10          /* a planning problem has no feasible point          */
 };
 
 enum { ANTDT_F32 = 0, ANTDT_BF16 = 1 };                  /* table row element type        */
@@ -135,6 +136,45 @@ int32_t antdt_dds_shard_info(const antdt_dds* dds, int64_t shard, int32_t* state
  * new handle.  CAPACITY if cap is too small, INVALID_ARG on a malformed image. */
 int32_t antdt_dds_save(const antdt_dds* dds, void* buf, size_t cap, size_t* used);
 int32_t antdt_dds_load(antdt_dds** out, const void* buf, size_t len);
+
+/* ---- controller front end (AntDT-ND, worker side) ------------------------------------ */
+enum { ANTDT_ACTION_NONE = 0, ANTDT_ACTION_ADJUST_BS = 1, ANTDT_ACTION_KILL_RESTART = 2 };
+typedef struct antdt_ctl antdt_ctl; /* opaque; host memory owned by the library */
+
+/* Section VI-A steps 2-5.  Keeps, per worker, the last window_trans and window_per reports
+ * (L^trans, L^per counted in reports), lambda = the slowness ratio (> 1; the paper uses 1.5).
+ * antdt_ctl_report: one (batch size, batch processing time in seconds) report of a worker.
+ * antdt_ctl_decide (every worker must have reported once, else STATE):
+ *   speeds[i]     v_i = mean over worker i's short window of batch_size / BPT of each report
+ *                 (the reading taken of the paper's throughput formula)
+ *   transient[i]  1 iff mean BPT over the short window >= lambda * (mean of those over workers)
+ *   persistent[i] the same over the long window
+ *   action        KILL_RESTART if any persistent straggler (the caller decides whether the
+ *                 cluster is busy), else ADJUST_BS if any transient one (feed `speeds` to
+ *                 antdt_shard_plan), else NONE.
+ * All arrays host [n_workers]. */
+int32_t antdt_ctl_create(antdt_ctl** out, int32_t n_workers, int32_t window_trans,
+                         int32_t window_per, double lambda);
+void antdt_ctl_destroy(antdt_ctl* ctl);
+int32_t antdt_ctl_report(antdt_ctl* ctl, int32_t worker, int64_t batch_size, double bpt_seconds);
+int32_t antdt_ctl_decide(const antdt_ctl* ctl, double* speeds, int32_t* transient,
+                         int32_t* persistent, int32_t* action);
+
+/* AntDT-DD, Section VI-B, Eq. 4 (its constraint read with the sum over the k device types):
+ *     min max_i C_i * B_i / v_i
+ *     s.t. sum_i n_i * C_i * B_i = B,  Bmin_i <= B_i <= Bmax_i,  Cmin <= C_i <= Cmax,
+ * all integers: device type i (n_i devices, throughput v_i) runs C_i accumulated micro-batches
+ * of B_i samples before the synchronisation.  Exact, by enumeration with pruning (k <= 8; meant
+ * for the handful of device types of a heterogeneous cluster); among equal optima the
+ * lexicographically smallest (C_1..C_k, B_1..B_k) is returned.  Each device of type i then
+ * enters the step with local batch C_i*B_i (accumulating C_i mean gradients of B_i samples is
+ * the mean over C_i*B_i samples, so the device path needs nothing else).
+ * Host arrays of n_types entries; z_out (may be NULL) receives the optimum.
+ * INFEASIBLE when no assignment meets the equality. */
+int32_t antdt_dd_solve(int32_t n_types, const int32_t* n_devices, const double* speeds,
+                       int64_t global_batch, const int64_t* batch_min, const int64_t* batch_max,
+                       int32_t accum_min, int32_t accum_max, int64_t* batch_out, int32_t* accum_out,
+                       double* z_out);
 
 /* ===================================================================================== */
 /* Device path                                                                           */

@@ -44,6 +44,10 @@ _lib.orc_aggregate_dense.argtypes = [_p, C.c_int64, C.c_int64, _p, C.c_int, _p]
 _lib.orc_sparse_opt_update.argtypes = [_p, C.c_int, C.c_int64, C.c_int, _p, _p, C.c_int64, C.c_int,
                                        C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64, _p, _p]
 
+_lib.orc_ctl_decide.argtypes = [_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_double, _p, _p, _p, _p]
+
+_lib.orc_dd_solve.argtypes = [C.c_int, _p, _p, C.c_int64, _p, _p, C.c_int, C.c_int, _p, _p, _p]
+
 RULES = {"proportional": 0, "minmax": 1}
 OPTS = {"adagrad": 0, "adam": 1}
 
@@ -185,3 +189,31 @@ def sparse_opt_update(table, ids, grads, opt, lr, eps, beta1, beta2, step, state
                                     _ptr(None if state1 is None else _chk(state1, _f32)))
     if rc:
         raise OracleError(rc)
+
+
+def ctl_decide(reports, K, Lt, Lp, lam):
+    """reports: rows (worker, batch size, BPT seconds) -> (speeds, transient, persistent, action)"""
+    r = np.ascontiguousarray(reports, dtype=_f64).reshape(-1, 3)
+    v = np.zeros(K, _f64)
+    t = np.zeros(K, np.int32)
+    p = np.zeros(K, np.int32)
+    a = C.c_int()
+    rc = _lib.orc_ctl_decide(_ptr(r), r.shape[0], K, Lt, Lp, lam, _ptr(v), _ptr(t), _ptr(p), C.byref(a))
+    if rc:
+        raise OracleError(rc)
+    return v, t, p, a.value
+
+
+def dd_solve(n_dev, v, B, bmin, bmax, cmin, cmax):
+    k = len(n_dev)
+    nd = np.ascontiguousarray(n_dev, dtype=np.int32)
+    vv = np.ascontiguousarray(v, dtype=_f64)
+    lo, hi = np.ascontiguousarray(bmin, dtype=_i64), np.ascontiguousarray(bmax, dtype=_i64)
+    b = np.zeros(k, _i64)
+    c = np.zeros(k, np.int32)
+    z = C.c_double()
+    rc = _lib.orc_dd_solve(k, _ptr(nd), _ptr(vv), B, _ptr(lo), _ptr(hi), cmin, cmax, _ptr(b), _ptr(c),
+                           C.byref(z))
+    if rc:
+        raise OracleError(rc)
+    return b, c, z.value

@@ -444,4 +444,84 @@ int orc_sparse_opt_update(void* table, int dtype, i64 n_rows, int dim, const i32
   return OK;
 }
 
+// AntDT-ND controller, worker side (Section VI-A steps 2-5), stateless form: the whole report
+// history is passed in.  reports: n_rep rows (worker, batch size, BPT seconds) in arrival order.
+// Window means over each worker's last Lt / Lp reports; straggler if mean_i >= lambda * mean over
+// workers; v_i = mean over the short window of batch / BPT.  action: 2 kill-restart if any
+// persistent, else 1 adjust-bs if any transient, else 0.
+int orc_ctl_decide(const double* reports, i64 n_rep, int K, int Lt, int Lp, double lambda,
+                   double* speeds, int* trans, int* pers, int* action) {
+  std::vector<std::vector<double> > bpt(K), rate(K);
+  for (i64 r = 0; r < n_rep; ++r) {
+    int w = (int)reports[3 * r];
+    if (w < 0 || w >= K || !(reports[3 * r + 2] > 0.0)) return E_ARG;
+    bpt[w].push_back(reports[3 * r + 2]);
+    rate[w].push_back(reports[3 * r + 1] / reports[3 * r + 2]);
+  }
+  std::vector<double> mt(K), mp(K);
+  double at = 0.0, ap = 0.0;
+  for (int i = 0; i < K; ++i) {
+    if (bpt[i].empty()) return 8;
+    size_t n = bpt[i].size();
+    size_t nt = std::min<size_t>(n, Lt), np_ = std::min<size_t>(n, Lp);
+    double s = 0.0, sr = 0.0, sp = 0.0;
+    for (size_t k = n - nt; k < n; ++k) { s += bpt[i][k]; sr += rate[i][k]; }
+    for (size_t k = n - np_; k < n; ++k) sp += bpt[i][k];
+    mt[i] = s / (double)nt;
+    speeds[i] = sr / (double)nt;
+    mp[i] = sp / (double)np_;
+    at += mt[i];
+    ap += mp[i];
+  }
+  at /= K;
+  ap /= K;
+  bool anyt = false, anyp = false;
+  for (int i = 0; i < K; ++i) {
+    trans[i] = mt[i] >= lambda * at;
+    pers[i] = mp[i] >= lambda * ap;
+    anyt = anyt || trans[i];
+    anyp = anyp || pers[i];
+  }
+  *action = anyp ? 2 : (anyt ? 1 : 0);
+  return OK;
+}
+
+// AntDT-DD, Eq. 4 (sum over the k device types): plain exhaustive search over every (C, B) in
+// lexicographic order of (C_1..C_k, B_1..B_k); the first strictly better point is kept, so ties
+// go to the lexicographically smallest.  Returns 10 when nothing is feasible.
+int orc_dd_solve(int k, const int* n_dev, const double* v, i64 B, const i64* bmin, const i64* bmax,
+                 int cmin, int cmax, i64* b_out, int* c_out, double* z_out) {
+  if (k < 1 || k > 8) return E_ARG;
+  std::vector<int> c(k, cmin);
+  bool found = false;
+  double best = 0.0;
+  for (;;) {  // odometer over C, last index fastest
+    std::vector<i64> b(bmin, bmin + k);
+    for (;;) {  // odometer over B, last index fastest
+      i64 total = 0;
+      double z = 0.0;
+      for (int i = 0; i < k; ++i) {
+        total += (i64)n_dev[i] * c[i] * b[i];
+        z = std::max(z, (double)(c[i] * b[i]) / v[i]);
+      }
+      if (total == B && (!found || z < best)) {
+        found = true;
+        best = z;
+        for (int i = 0; i < k; ++i) { b_out[i] = b[i]; c_out[i] = c[i]; }
+      }
+      int i = k - 1;
+      while (i >= 0 && b[i] == bmax[i]) { b[i] = bmin[i]; --i; }
+      if (i < 0) break;
+      b[i] += 1;
+    }
+    int i = k - 1;
+    while (i >= 0 && c[i] == cmax) { c[i] = cmin; --i; }
+    if (i < 0) break;
+    c[i] += 1;
+  }
+  if (!found) return 10;
+  *z_out = best;
+  return OK;
+}
+
 }  // extern "C"

@@ -13,7 +13,7 @@ from typing import Optional, Sequence
 import torch
 
 OK, ERR_INVALID_ARG, ERR_ID_OUT_OF_RANGE, ERR_WORKSPACE_TOO_SMALL, ERR_CAPACITY, ERR_CUDA, \
-    ERR_TIMEOUT, ERR_EXHAUSTED, ERR_STATE, ERR_BAD_OFFSETS = range(10)
+    ERR_TIMEOUT, ERR_EXHAUSTED, ERR_STATE, ERR_BAD_OFFSETS, ERR_INFEASIBLE = range(11)
 F32, BF16 = 0, 1
 RULE_PROPORTIONAL, RULE_MINMAX = 0, 1
 OPT_ADAGRAD, OPT_ADAM = 0, 1
@@ -27,7 +27,8 @@ _lib = None
 EXPORTS = [
     "antdt_dds_create", "antdt_dds_destroy", "antdt_batch_sizes", "antdt_shard_plan",
     "antdt_dds_requeue_worker", "antdt_dds_num_shards", "antdt_dds_counts", "antdt_dds_shard_info",
-    "antdt_dds_save", "antdt_dds_load", "antdt_embbag_fwd",
+    "antdt_dds_save", "antdt_dds_load", "antdt_ctl_create", "antdt_ctl_destroy",
+    "antdt_ctl_report", "antdt_ctl_decide", "antdt_dd_solve", "antdt_embbag_fwd",
     "antdt_embbag_bwd_dedup_workspace_bytes", "antdt_embbag_bwd_dedup",
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
@@ -103,6 +104,13 @@ def lib() -> C.CDLL:
         L.antdt_dds_shard_info.argtypes = [P, I64, P, P, P]
         L.antdt_dds_save.argtypes = [P, P, SZ, C.POINTER(SZ)]
         L.antdt_dds_load.argtypes = [C.POINTER(P), P, SZ]
+        L.antdt_ctl_create.argtypes = [C.POINTER(P), I32, I32, I32, D]
+        L.antdt_ctl_destroy.argtypes = [P]
+        L.antdt_ctl_destroy.restype = None
+        L.antdt_ctl_report.argtypes = [P, I32, I64, D]
+        L.antdt_ctl_decide.argtypes = [P, P, P, P, P]
+        L.antdt_dd_solve.argtypes = [I32, P, P, I64, P, P, I32, I32, P, P, P]
+        L.antdt_dd_solve.restype = I32
         L.antdt_embbag_fwd.argtypes = [P, I32, I64, I32, P, I64, P, I64, P, P, P]
         L.antdt_embbag_bwd_dedup_workspace_bytes.argtypes = [I64, I64, I32, I32]
         L.antdt_embbag_bwd_dedup_workspace_bytes.restype = SZ
@@ -122,9 +130,11 @@ def lib() -> C.CDLL:
         L.antdt_profile_enable.argtypes = [I32]
         L.antdt_profile_get.argtypes = [I32, C.c_char_p, SZ, C.POINTER(I64), C.POINTER(D)]
         L.antdt_version.restype = C.c_char_p
-        for fn in ("antdt_dds_create", "antdt_batch_sizes", "antdt_shard_plan",
+        for fn in ("antdt_ctl_create", "antdt_ctl_report", "antdt_ctl_decide",
+                   "antdt_dds_create", "antdt_batch_sizes", "antdt_shard_plan",
                    "antdt_dds_requeue_worker", "antdt_dds_counts", "antdt_dds_shard_info",
-                   "antdt_dds_save", "antdt_dds_load", "antdt_embbag_fwd", "antdt_embbag_bwd_dedup",
+                   "antdt_dds_save", "antdt_dds_load", "antdt_ctl_create", "antdt_ctl_destroy",
+    "antdt_ctl_report", "antdt_ctl_decide", "antdt_dd_solve", "antdt_embbag_fwd", "antdt_embbag_bwd_dedup",
                    "antdt_weighted_aggregate", "antdt_sparse_opt_update", "antdt_bsp_step_host",
                    "antdt_read_status", "antdt_profile_enable", "antdt_profile_kernels",
                    "antdt_profile_get"):
@@ -240,6 +250,47 @@ class Dds:
         h = C.c_void_p()
         _check(lib().antdt_dds_load(C.byref(h), image, len(image)), "antdt_dds_load")
         return Dds(0, 0, 0, n_workers, _handle=h)
+
+
+ACTION_NONE, ACTION_ADJUST_BS, ACTION_KILL_RESTART = 0, 1, 2
+
+
+class Ctl:
+    """Handle of the AntDT-ND controller front end (antdt_ctl_* calls)."""
+
+    def __init__(self, n_workers: int, window_trans: int, window_per: int, lam: float):
+        self.K = n_workers
+        h = C.c_void_p()
+        _check(lib().antdt_ctl_create(C.byref(h), n_workers, window_trans, window_per, lam),
+               "antdt_ctl_create")
+        self._h = h
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib().antdt_ctl_destroy(self._h)
+            self._h = None
+
+    def antdt_ctl_report(self, worker: int, batch_size: int, bpt_seconds: float):
+        _check(lib().antdt_ctl_report(self._h, worker, batch_size, bpt_seconds), "antdt_ctl_report")
+
+    def antdt_ctl_decide(self):
+        """-> (speeds [K], transient [K], persistent [K], action)"""
+        K = self.K
+        v, t, p, a = (C.c_double * K)(), (C.c_int32 * K)(), (C.c_int32 * K)(), C.c_int32()
+        _check(lib().antdt_ctl_decide(self._h, v, t, p, C.byref(a)), "antdt_ctl_decide")
+        return list(v), list(t), list(p), a.value
+
+
+def antdt_dd_solve(n_devices, speeds, global_batch: int, batch_min, batch_max, accum_min: int,
+                   accum_max: int):
+    """-> (B_i list, C_i list, z) of Eq. 4; raises AntdtError(ERR_INFEASIBLE) if there is none."""
+    k = len(n_devices)
+    nd = (C.c_int32 * k)(*[int(x) for x in n_devices])
+    b, c, z = (C.c_int64 * k)(), (C.c_int32 * k)(), C.c_double()
+    _check(lib().antdt_dd_solve(k, nd, _f64s(speeds), global_batch, _i64s(batch_min),
+                                _i64s(batch_max), accum_min, accum_max, b, c, C.byref(z)),
+           "antdt_dd_solve")
+    return list(b), list(c), z.value
 
 
 # ---- device path ---------------------------------------------------------------------------
