@@ -287,6 +287,18 @@ int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_
                                  const int64_t* batch_sizes, int32_t n_workers, void* ws,
                                  size_t ws_bytes, int32_t* dev_status, void* stream);
 
+/* Backup-workers variant of the aggregation (the replication-based baseline the paper compares
+ * with, Section VII-A.3: the gradients of the b slowest workers are disregarded in an iteration
+ * and their samples go back to the shard service, antdt_dds_requeue_worker).  dropped: host
+ * [K], non-zero = this worker's lists and dense vector are ignored altogether: rows that only
+ * dropped workers touched are not in agg_ids, and the weights are b_i / sum over the SURVIVING
+ * workers' b_j, so the result is the mean gradient over the samples that count.  Everything
+ * else as antdt_weighted_aggregate (same workspace size). */
+int32_t antdt_weighted_aggregate_backup(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                        const int64_t* batch_sizes, const uint8_t* dropped,
+                                        int32_t n_workers, void* ws, size_t ws_bytes,
+                                        int32_t* dev_status, void* stream);
+
 /* Server update (Section II: the servers "update the parameters"), on the rows in ids only;
  * every other row of table and state is left bit-identical.
  *   Adagrad: state0 += g*g;  w -= lr * g / (sqrt(state0) + eps)

@@ -48,6 +48,10 @@ _lib.orc_ctl_decide.argtypes = [_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_do
 
 _lib.orc_dd_solve.argtypes = [C.c_int, _p, _p, C.c_int64, _p, _p, C.c_int, C.c_int, _p, _p, _p]
 
+_lib.orc_aggregate_sparse_backup.restype = C.c_int64
+_lib.orc_aggregate_sparse_backup.argtypes = [C.c_int, _p, _p, _p, _p, _p, C.c_int, _p, _p, C.c_int64]
+_lib.orc_aggregate_dense_backup.argtypes = [_p, C.c_int64, C.c_int64, _p, _p, C.c_int, _p]
+
 RULES = {"proportional": 0, "minmax": 1}
 OPTS = {"adagrad": 0, "adam": 1}
 
@@ -217,3 +221,30 @@ def dd_solve(n_dev, v, B, bmin, bmax, cmin, cmax):
     if rc:
         raise OracleError(rc)
     return b, c, z.value
+
+
+def aggregate_sparse_backup(uniq_ids, worker_uniq_offsets, uniq_grads, batch_sizes_, dropped):
+    K = worker_uniq_offsets.shape[0] - 1
+    n = int(worker_uniq_offsets[K])
+    D = uniq_grads.shape[1]
+    ids = np.zeros(max(n, 1), _i32)
+    g = np.zeros((max(n, 1), D), _f32)
+    d = np.ascontiguousarray(dropped, dtype=np.uint8)
+    na = _lib.orc_aggregate_sparse_backup(D, _ptr(_chk(uniq_ids, _i32)), _ptr(_chk(worker_uniq_offsets, _i64)),
+                                          _ptr(_chk(uniq_grads, _f32)),
+                                          _ptr(np.ascontiguousarray(batch_sizes_, _i64)), _ptr(d), K,
+                                          _ptr(ids), _ptr(g), max(n, 1))
+    if na < 0:
+        raise OracleError(-na)
+    return ids[:na].copy(), g[:na].copy()
+
+
+def aggregate_dense_backup(grads, batch_sizes_, dropped):
+    K, n = grads.shape
+    out = np.zeros(n, _f32)
+    d = np.ascontiguousarray(dropped, dtype=np.uint8)
+    rc = _lib.orc_aggregate_dense_backup(_ptr(_chk(grads, _f32)), n, n,
+                                         _ptr(np.ascontiguousarray(batch_sizes_, _i64)), _ptr(d), K, _ptr(out))
+    if rc:
+        raise OracleError(rc)
+    return out

@@ -524,4 +524,52 @@ int orc_dd_solve(int k, const int* n_dev, const double* v, i64 B, const i64* bmi
   return OK;
 }
 
+// Backup-workers aggregation (Section VII-A.3): the dropped workers do not exist for this step.
+// Union and weights over the surviving workers only, w_i = b_i / sum_{surviving} b_j.
+i64 orc_aggregate_sparse_backup(int dim, const i32* uniq_ids, const i64* wuo, const float* uniq_grads,
+                                const i64* bsz, const uint8_t* dropped, int K, i32* agg_ids,
+                                float* agg_grads, i64 cap) {
+  double tot = 0.0;
+  for (int i = 0; i < K; ++i)
+    if (!dropped[i]) tot += (double)bsz[i];
+  if (!(tot > 0.0)) return -E_ARG;
+  std::vector<i32> all;
+  for (int i = 0; i < K; ++i)
+    if (!dropped[i]) all.insert(all.end(), uniq_ids + wuo[i], uniq_ids + wuo[i + 1]);
+  std::sort(all.begin(), all.end());
+  all.erase(std::unique(all.begin(), all.end()), all.end());
+  if ((i64)all.size() > cap) return -E_CAP;
+  for (size_t u = 0; u < all.size(); ++u) {
+    agg_ids[u] = all[u];
+    std::vector<double> s(dim, 0.0);
+    for (int i = 0; i < K; ++i) {
+      if (dropped[i]) continue;
+      const i32* lo = uniq_ids + wuo[i];
+      const i32* hi = uniq_ids + wuo[i + 1];
+      const i32* it = std::lower_bound(lo, hi, all[u]);
+      if (it == hi || *it != all[u]) continue;
+      double wi = (double)bsz[i] / tot;
+      const float* g = uniq_grads + (i64)(it - uniq_ids) * dim;
+      for (int c = 0; c < dim; ++c) s[c] += wi * (double)g[c];
+    }
+    for (int c = 0; c < dim; ++c) agg_grads[(i64)u * dim + c] = (float)s[c];
+  }
+  return (i64)all.size();
+}
+
+int orc_aggregate_dense_backup(const float* grads, i64 n, i64 stride, const i64* bsz,
+                               const uint8_t* dropped, int K, float* out) {
+  double tot = 0.0;
+  for (int i = 0; i < K; ++i)
+    if (!dropped[i]) tot += (double)bsz[i];
+  if (!(tot > 0.0)) return E_ARG;
+  for (i64 e = 0; e < n; ++e) {
+    double s = 0.0;
+    for (int i = 0; i < K; ++i)
+      if (!dropped[i]) s += ((double)bsz[i] / tot) * (double)grads[(i64)i * stride + e];
+    out[e] = (float)s;
+  }
+  return OK;
+}
+
 }  // extern "C"

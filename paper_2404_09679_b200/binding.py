@@ -32,6 +32,7 @@ EXPORTS = [
     "antdt_embbag_bwd_dedup_workspace_bytes", "antdt_embbag_bwd_dedup",
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
+    "antdt_weighted_aggregate_backup",
     "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_read_status", "antdt_launch_count",
     "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_version",
 ]
@@ -122,6 +123,8 @@ def lib() -> C.CDLL:
         L.antdt_weighted_aggregate_workspace_bytes.argtypes = [I64, I32, I32]
         L.antdt_weighted_aggregate_workspace_bytes.restype = SZ
         L.antdt_weighted_aggregate.argtypes = [P, P, P, I32, P, SZ, P, P]
+        L.antdt_weighted_aggregate_backup.argtypes = [P, P, P, P, I32, P, SZ, P, P]
+        L.antdt_weighted_aggregate_backup.restype = I32
         L.antdt_sparse_opt_update.argtypes = [P, I32, I64, I32, P, P, P, I64, I32, F, F, F, F, I64,
                                               P, P, P, P]
         L.antdt_bsp_step_host.argtypes = [P, P]
@@ -345,8 +348,9 @@ def antdt_weighted_aggregate_workspace_bytes(in_cap: int, dim: int, n_workers: i
 def antdt_weighted_aggregate(batch_sizes: Sequence[int], ws, *, n_rows: int = 0, uniq_ids=None,
                              worker_uniq_offsets=None, uniq_grads=None, agg_ids=None,
                              agg_grads=None, n_agg=None, dense_grads=None, dense_out=None,
-                             dev_status=None, stream=None):
-    """Sparse part when uniq_ids is given, dense part when dense_grads ([K, n]) is given."""
+                             dev_status=None, stream=None, dropped=None):
+    """Sparse part when uniq_ids is given, dense part when dense_grads ([K, n]) is given.
+    dropped (list of K flags) selects antdt_weighted_aggregate_backup."""
     K = len(batch_sizes)
     sp = dp = None
     if uniq_ids is not None:
@@ -357,6 +361,13 @@ def antdt_weighted_aggregate(batch_sizes: Sequence[int], ws, *, n_rows: int = 0,
     if dense_grads is not None:
         dp = DensePart(dense_grads.data_ptr(), dense_grads.shape[1], dense_grads.stride(0),
                        dense_out.data_ptr())
+    if dropped is not None:
+        flags = (C.c_uint8 * K)(*[1 if d else 0 for d in dropped])
+        _check(lib().antdt_weighted_aggregate_backup(
+            C.byref(sp) if sp else None, C.byref(dp) if dp else None, _i64s(batch_sizes), flags, K,
+            _dp(ws), ws.numel() * ws.element_size(), _dp(dev_status), _stream(stream)),
+            "antdt_weighted_aggregate_backup")
+        return
     _check(lib().antdt_weighted_aggregate(
         C.byref(sp) if sp else None, C.byref(dp) if dp else None, _i64s(batch_sizes), K, _dp(ws),
         ws.numel() * ws.element_size(), _dp(dev_status), _stream(stream)),

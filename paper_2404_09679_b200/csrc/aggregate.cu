@@ -17,7 +17,7 @@ size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct AggLayout {
   SortLayout sort;
-  size_t sort_ws, bounds, weights, wuo, keys_a, keys_b, src, vals_t, run_start, head_bits,
+  size_t sort_ws, bounds, weights, wuo, cwuo, drop, keys_a, keys_b, src, vals_t, run_start, head_bits,
       tile_first, head_part, tail_part, bytes;
 };
 
@@ -30,6 +30,8 @@ AggLayout agg_layout(int64_t in_cap, int K, int dim) {
   L.bounds = o;    o = align_up(o + 16);
   L.weights = o;   o = align_up(o + 4 * (size_t)K);
   L.wuo = o;       o = align_up(o + 8 * ((size_t)K + 1));
+  L.cwuo = o;      o = align_up(o + 8 * ((size_t)K + 1));
+  L.drop = o;      o = align_up(o + 4 * (size_t)K);
   L.keys_a = o;    o = align_up(o + 4 * n);
   L.keys_b = o;    o = align_up(o + 4 * n);
   L.src = o;       o = align_up(o + 4 * n);
@@ -66,7 +68,58 @@ __global__ void agg_prep_kernel(const int64_t* __restrict__ wuo_in, int K, int64
   }
 }
 
-// dense_out[e] = sum_i w_i * g_i[e], ascending i, one float4 per thread
+// Backup-workers variant: only the surviving workers' lists are merged.  prep computes where
+// each survivor's list starts in the compacted concatenation, compact copies (row id, original
+// position) of the survivors' entries there; the original position stays the payload, so the
+// reduction finds rows and weights exactly as in the plain variant.
+__global__ void agg_prep_backup_kernel(const int64_t* __restrict__ wuo_in, const uint32_t* __restrict__ drop,
+                                       int K, int64_t in_cap, int64_t* __restrict__ bounds,
+                                       int64_t* __restrict__ wuo, int64_t* __restrict__ cwuo,
+                                       int32_t* status) {
+  if (threadIdx.x != 0) return;
+  int64_t prev = 0, acc = 0;
+  for (int i = 0; i <= K; ++i) {  // K <= 1024: a serial pass is enough
+    int64_t v = wuo_in[i];
+    v = v < prev ? prev : v;
+    v = v > in_cap ? in_cap : v;
+    wuo[i] = v;
+    if (i > 0) {
+      cwuo[i - 1] = acc;
+      if (!drop[i - 1]) acc += v - prev;
+    }
+    prev = v;
+  }
+  cwuo[K] = acc;
+  if (wuo_in[K] < 0 || wuo_in[K] > in_cap) set_status(status, ANTDT_ERR_CAPACITY);
+  bounds[0] = 0;
+  bounds[1] = acc;
+}
+
+__global__ void __launch_bounds__(256)
+agg_compact_kernel(const int32_t* __restrict__ uniq_ids, const int64_t* __restrict__ wuo,
+                   const int64_t* __restrict__ cwuo, const uint32_t* __restrict__ drop, int K,
+                   uint32_t* __restrict__ keys_c, uint32_t* __restrict__ vals_c) {
+  extern __shared__ int64_t s_cw[];  // wuo [K+1], cwuo [K+1], then K drop flags
+  int64_t* s_wuo = s_cw;
+  int64_t* s_cwuo = s_cw + (K + 1);
+  uint32_t* s_drop = reinterpret_cast<uint32_t*>(s_cw + 2 * (K + 1));
+  for (int i = threadIdx.x; i <= K; i += blockDim.x) { s_wuo[i] = wuo[i]; s_cwuo[i] = cwuo[i]; }
+  for (int i = threadIdx.x; i < K; i += blockDim.x) s_drop[i] = drop[i];
+  __syncthreads();
+  const int64_t n = s_wuo[K];
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += step) {
+    int w = interval_of(s_wuo, K + 1, p);
+    if (w > K - 1) w = K - 1;
+    if (s_drop[w]) continue;
+    const int64_t dst = s_cwuo[w] + (p - s_wuo[w]);
+    keys_c[dst] = (uint32_t)uniq_ids[p];
+    vals_c[dst] = (uint32_t)p;
+  }
+}
+
+// dense_out[e] = sum_i w_i * g_i[e], ascending i, one float4 per thread; a worker of weight 0
+// (empty or dropped) is not read at all
 __global__ void __launch_bounds__(256)
 dense_wsum_kernel(const float* __restrict__ grads, int64_t n4, int64_t stride,
                   const float* __restrict__ weights, int K, float* __restrict__ out) {
@@ -81,7 +134,8 @@ dense_wsum_kernel(const float* __restrict__ grads, int64_t n4, int64_t stride,
     for (; i + 4 <= K; i += 4) {
       float4 v[4];
 #pragma unroll
-      for (int t = 0; t < 4; ++t) v[t] = ldg_f4(p + (size_t)(i + t) * stride);
+      for (int t = 0; t < 4; ++t)
+        v[t] = s_wd[i + t] != 0.f ? ldg_f4(p + (size_t)(i + t) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const float w = s_wd[i + t];
@@ -90,8 +144,9 @@ dense_wsum_kernel(const float* __restrict__ grads, int64_t n4, int64_t stride,
       }
     }
     for (; i < K; ++i) {
-      const float4 v = ldg_f4(p + (size_t)i * stride);
       const float w = s_wd[i];
+      if (w == 0.f) continue;
+      const float4 v = ldg_f4(p + (size_t)i * stride);
       acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
       acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
     }
@@ -109,16 +164,20 @@ extern "C" size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32
   return antdt::agg_layout(in_cap, n_workers, dim).bytes;
 }
 
-extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,
-                                            const int64_t* batch_sizes, int32_t n_workers, void* ws,
-                                            size_t ws_bytes, int32_t* dev_status, void* stream) {
-  using namespace antdt;
+namespace antdt {
+namespace {
+int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                       const int64_t* batch_sizes, const uint8_t* dropped, int32_t n_workers,
+                       void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
   const int K = n_workers;
   if (K < 1 || K > kMaxSegments || !batch_sizes || !ws || !aligned16(ws)) return ANTDT_ERR_INVALID_ARG;
   double tot = 0.0;
+  bool any_dropped = false;
   for (int i = 0; i < K; ++i) {
     if (batch_sizes[i] < 0) return ANTDT_ERR_INVALID_ARG;
-    tot += (double)batch_sizes[i];
+    const bool d = dropped && dropped[i];
+    any_dropped |= d;
+    if (!d) tot += (double)batch_sizes[i];
   }
   if (!(tot > 0.0)) return ANTDT_ERR_INVALID_ARG;
   const int64_t in_cap = sp ? sp->in_cap : 0;
@@ -143,19 +202,46 @@ extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const a
 
   // w_i = b_i / sum_j b_j, formed in double, used in fp32
   float hw[kMaxSegments];
-  for (int i = 0; i < K; ++i) hw[i] = (float)((double)batch_sizes[i] / tot);
+  for (int i = 0; i < K; ++i)
+    hw[i] = (dropped && dropped[i]) ? 0.f : (float)((double)batch_sizes[i] / tot);
   upload_small(hw, 4 * (size_t)K, w8 + L.weights, s);
 
   if (sp) {
     char* sort_ws = w8 + L.sort_ws;
     int64_t* bounds = (int64_t*)(w8 + L.bounds);
     uint32_t* keys_a = (uint32_t*)(w8 + L.keys_a);
-    ANTDT_LAUNCH("agg_prep", agg_prep_kernel, 1, 256, 0, s, sp->worker_uniq_offsets, K, in_cap,
-                 bounds, (int64_t*)(w8 + L.wuo), dev_status);
+    const uint32_t* sort_keys = reinterpret_cast<const uint32_t*>(sp->uniq_ids);
+    const uint32_t* sort_vals = nullptr;  // payload = position in the concatenated lists
+    const int key_bits = bits_for(sp->n_rows);
+    if (!any_dropped) {
+      ANTDT_LAUNCH("agg_prep", agg_prep_kernel, 1, 256, 0, s, sp->worker_uniq_offsets, K, in_cap,
+                   bounds, (int64_t*)(w8 + L.wuo), dev_status);
+    } else {
+      uint32_t hd[kMaxSegments];
+      for (int i = 0; i < K; ++i) hd[i] = dropped[i] ? 1u : 0u;
+      uint32_t* d_drop = (uint32_t*)(w8 + L.drop);
+      int64_t* cwuo = (int64_t*)(w8 + L.cwuo);
+      upload_small(hd, 4 * (size_t)K, d_drop, s);
+      ANTDT_LAUNCH("agg_prep", agg_prep_backup_kernel, 1, 32, 0, s, sp->worker_uniq_offsets, d_drop,
+                   K, in_cap, bounds, (int64_t*)(w8 + L.wuo), cwuo, dev_status);
+      // the compacted input lives in the pair of sort buffers that the first pass does not
+      // write: the temporaries when the pass count is odd, the outputs when it is even
+      const bool odd = sort_passes(key_bits) % 2 == 1;
+      uint32_t* keys_c = (uint32_t*)(w8 + (odd ? L.keys_b : L.keys_a));
+      uint32_t* vals_c = (uint32_t*)(w8 + (odd ? L.vals_t : L.src));
+      if (in_cap > 0) {
+        int64_t want = (in_cap + 255) / 256;
+        const int64_t gcap = (int64_t)kNumSM * 16;
+        ANTDT_LAUNCH("agg_compact", agg_compact_kernel, (unsigned)(want > gcap ? gcap : want), 256,
+                     16 * ((size_t)K + 1) + 4 * (size_t)K, s, sp->uniq_ids,
+                     (const int64_t*)(w8 + L.wuo), cwuo, d_drop, K, keys_c, vals_c);
+      }
+      sort_keys = keys_c;
+      sort_vals = vals_c;
+    }
     segsort_setup(bounds, 1, in_cap, sort_ws, L.sort, s);
-    segsort_run(reinterpret_cast<const uint32_t*>(sp->uniq_ids), nullptr, keys_a,
-                (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b), (uint32_t*)(w8 + L.vals_t),
-                bits_for(sp->n_rows), 0, sort_ws, L.sort, dev_status, s, true);
+    segsort_run(sort_keys, sort_vals, keys_a, (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b),
+                (uint32_t*)(w8 + L.vals_t), key_bits, 0, sort_ws, L.sort, dev_status, s, true);
     segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
                  sp->out_cap < in_cap ? sp->out_cap : in_cap, (uint32_t*)(w8 + L.head_bits),
                  (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s, true);
@@ -188,4 +274,23 @@ extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const a
                  dp->stride, (const float*)(w8 + L.weights), K, dp->out);
   }
   return cuda_ok();
+}
+}  // namespace
+}  // namespace antdt
+
+extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                            const int64_t* batch_sizes, int32_t n_workers, void* ws,
+                                            size_t ws_bytes, int32_t* dev_status, void* stream) {
+  return antdt::aggregate_impl(sp, dp, batch_sizes, nullptr, n_workers, ws, ws_bytes, dev_status,
+                               stream);
+}
+
+extern "C" int32_t antdt_weighted_aggregate_backup(const antdt_sparse_part* sp,
+                                                   const antdt_dense_part* dp,
+                                                   const int64_t* batch_sizes, const uint8_t* dropped,
+                                                   int32_t n_workers, void* ws, size_t ws_bytes,
+                                                   int32_t* dev_status, void* stream) {
+  if (!dropped) return ANTDT_ERR_INVALID_ARG;
+  return antdt::aggregate_impl(sp, dp, batch_sizes, dropped, n_workers, ws, ws_bytes, dev_status,
+                               stream);
 }

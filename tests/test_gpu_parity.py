@@ -323,3 +323,38 @@ def test_dense_part_alone_and_sparse_part_alone():
     B.antdt_weighted_aggregate([int(b) for b in bsz], ws, dense_grads=wide[:, :n], dense_out=out,
                                dev_status=st)
     G.close(out.cpu().numpy(), oracle.aggregate_dense(g, bsz))
+
+
+def test_backup_workers_aggregate_matches_checker():
+    rng = np.random.default_rng(43)
+    for V, D, K, n_per in [(500, 16, 6, 300), (200_000, 64, 16, 20_000), (3000, 32, 33, 500)]:
+        lists = [np.sort(rng.choice(V, size=int(rng.integers(1, n_per + 1)), replace=False))
+                 for _ in range(K)]
+        uid = np.concatenate(lists).astype(np.int32)
+        wuo = np.concatenate([[0], np.cumsum([len(l) for l in lists])]).astype(np.int64)
+        g = rng.normal(size=(len(uid), D)).astype(np.float32)
+        bsz = rng.integers(1, 5000, size=K)
+        dropped = (rng.random(K) < 0.3).astype(np.uint8)
+        dropped[0], dropped[1] = 1, 0
+        dense = (1e-2 * rng.normal(size=(K, 4096))).astype(np.float32)
+        dense[0] = np.nan                                # a dropped worker's vector is never read
+        cap = len(uid)
+        agg_ids = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
+        agg = torch.full((cap, D), float("nan"), device="cuda")
+        n_agg = torch.zeros(1, dtype=torch.int64, device="cuda")
+        dout = torch.full((4096,), float("nan"), device="cuda")
+        ws = torch.empty(B.antdt_weighted_aggregate_workspace_bytes(cap, D, K), dtype=torch.uint8,
+                         device="cuda")
+        st = G.new_status()
+        B.antdt_weighted_aggregate([int(b) for b in bsz], ws, n_rows=V, uniq_ids=G.dev(uid),
+                                   worker_uniq_offsets=G.dev(wuo), uniq_grads=G.dev(g),
+                                   agg_ids=agg_ids, agg_grads=agg, n_agg=n_agg,
+                                   dense_grads=G.dev(dense), dense_out=dout, dev_status=st,
+                                   dropped=dropped.tolist())
+        assert B.antdt_read_status(st) == 0
+        want_ids, want = oracle.aggregate_sparse_backup(uid, wuo, g, bsz, dropped)
+        na = int(n_agg.item())
+        assert na == len(want_ids) and np.array_equal(agg_ids[:na].cpu().numpy(), want_ids)
+        G.close(agg[:na].cpu().numpy(), want)
+        dense[0] = 0
+        G.close(dout.cpu().numpy(), oracle.aggregate_dense_backup(dense, bsz, dropped))

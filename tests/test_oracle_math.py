@@ -254,3 +254,33 @@ def test_update_rejects_out_of_range_id():
     with pytest.raises(oracle.OracleError):
         oracle.sparse_opt_update(W, np.array([3], np.int32), np.zeros((1, 4), np.float32),
                                  "adagrad", 0.01, 1e-8, 0, 0, 1, np.zeros((3, 4), np.float32))
+
+
+# ---- backup-workers aggregation --------------------------------------------------------------
+def test_backup_aggregate_is_the_mean_over_the_surviving_samples():
+    rng = np.random.default_rng(40)
+    V, D, F, K, S = 60, 4, 3, 5, 40
+    ids, off = random_bags(rng, S * F, V, 4, zipf=1.3)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    wso = np.array([0, 3, 11, 20, 30, S], np.int64)
+    bsz = np.diff(wso)
+    dropped = np.array([0, 1, 0, 0, 1], np.uint8)            # workers 1 and 4 are the slowest
+    r = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+    agg_ids, agg = oracle.aggregate_sparse_backup(r["uniq_ids"], r["worker_uniq_offsets"],
+                                                  r["uniq_grads"], bsz, dropped)
+    # forget workers: mean gradient over the samples of workers 0, 2, 3 only
+    keep_bags = np.concatenate([np.arange(wso[w] * F, wso[w + 1] * F) for w in (0, 2, 3)])
+    A = count_matrix(ids, off, V)[keep_bags]
+    full = A.T @ dY[keep_bags].astype(np.float64) / float(bsz[[0, 2, 3]].sum())
+    rows = np.flatnonzero(A.sum(0))
+    assert np.array_equal(agg_ids, rows.astype(np.int32))
+    assert np.allclose(agg, full[rows], rtol=2e-6, atol=1e-8)
+    # nobody dropped: the plain aggregate, bit for bit
+    a0, g0 = oracle.aggregate_sparse_backup(r["uniq_ids"], r["worker_uniq_offsets"], r["uniq_grads"],
+                                            bsz, np.zeros(K, np.uint8))
+    a1, g1 = oracle.aggregate_sparse(r["uniq_ids"], r["worker_uniq_offsets"], r["uniq_grads"], bsz)
+    assert np.array_equal(a0, a1) and np.array_equal(g0, g1)
+    dense = rng.normal(size=(K, 16)).astype(np.float32)
+    d = oracle.aggregate_dense_backup(dense, bsz, dropped)
+    w = bsz[[0, 2, 3]] / bsz[[0, 2, 3]].sum()
+    assert np.allclose(d, (w[:, None] * dense[[0, 2, 3]].astype(np.float64)).sum(0), rtol=1e-6, atol=1e-9)
