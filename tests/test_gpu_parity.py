@@ -358,3 +358,26 @@ def test_backup_workers_aggregate_matches_checker():
         G.close(agg[:na].cpu().numpy(), want)
         dense[0] = 0
         G.close(dout.cpu().numpy(), oracle.aggregate_dense_backup(dense, bsz, dropped))
+
+
+def test_bwd_extreme_row_ids_and_widest_rows():
+    # row ids up to 2^31 - 2: 31-bit keys, four radix passes (nothing here touches a table)
+    rng = np.random.default_rng(44)
+    V, D, K, F, S = (1 << 31) - 1, 8, 3, 2, 4000
+    ids = rng.integers(V - 5000, V, size=S * F * 2).astype(np.int32)
+    ids[::7] = rng.integers(0, 50, size=len(ids[::7]))           # and some at the low end
+    off = np.arange(0, S * F * 2 + 1, 2, dtype=np.int64)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    _check_bwd(ids, off, F, dY, V, _wso(rng, K, S))
+    # dim 1024: eight vectors per lane
+    V, D, S = 300, 1024, 200
+    ids, off = random_bags(rng, S * F, V, 3, zipf=1.2)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    got, want = _check_bwd(ids, off, F, dY, V, _wso(rng, K, S))
+    bsz = np.maximum(np.diff(_wso(rng, K, S)), 1)
+    aid, agg, na, _, code = G.gpu_aggregate(got["uniq_ids"], got["worker_uniq_offsets"],
+                                            got["uniq_grads"], bsz, V)
+    wid, wagg = oracle.aggregate_sparse(want["uniq_ids"], want["worker_uniq_offsets"],
+                                        want["uniq_grads"], bsz)
+    assert code == 0 and np.array_equal(aid, wid)
+    G.close(agg, wagg, rtol=3e-5, atol=2e-6)
