@@ -10,7 +10,7 @@
 namespace antdt {
 namespace {
 
-constexpr int kFwdThreads = 256;
+constexpr int kFwdThreads = 128;
 constexpr int kFwdUnroll = 4;
 
 template <int G, int VPL, bool BF16>
