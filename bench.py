@@ -277,7 +277,7 @@ def cpu_baseline(w, cfg, bm, plan, table):
 def run_ours(args):
     from paper_2404_09679_b200 import binding as B
     from paper_2404_09679_b200 import synth
-    from paper_2404_09679_b200.step import OptConfig, StepBuffers, run_step
+    from paper_2404_09679_b200.step import DeviceStep, OptConfig, StepBuffers
 
     rank, local_rank, world = dist_setup("nccl")
     if not torch.cuda.is_available():
@@ -332,6 +332,7 @@ def run_ours(args):
     buf = StepBuffers(w.D, w.K, max_nnz, max_bags, w.dense_n, uniq_cap=cap, agg_cap=cap, device=dev)
 
     dds = B.Dds(w.n_samples, w.B, w.M, w.K)                # the live planner of the timed loop
+    dstep = DeviceStep(buf, table, state0, state1, oc, w.K)  # the four device calls behind one C call
 
     def one_step(s):
         b = batches[s % n_batches]
@@ -339,8 +340,7 @@ def run_ours(args):
         rc, bsz, _, _, cnt = dds.antdt_shard_plan(v, B.RULES[w.rule], w.min_batch)
         if s < len(plans):
             assert rc == B.OK and cnt == plans[s]["counts"]
-        run_step(buf, table, state0, state1, oc, s + 1, b["ids"], b["off"], w.F, b["dY"], b["wso"],
-                 b["counts"], b["dense"])
+        dstep.run(s + 1, b["ids"], b["off"], w.F, b["dY"], b["wso"], b["counts"], b["dense"])
 
     stream = torch.cuda.current_stream()
     for s in range(W):

@@ -350,6 +350,11 @@ typedef struct {
   int64_t* h_n_agg; int32_t* h_status;  /* one element each                                */
 } antdt_step_desc;
 int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream);
+/* The same step for a batch that already sits in device memory: the d_row_ids, d_bag_offsets,
+ * d_d_pooled and d_dense_grads fields of the descriptor are the inputs, every h_* field is
+ * ignored, nothing is copied, and the status word is neither cleared nor read back.  One host
+ * call instead of four: for small batches the per-call host cost is the step time. */
+int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream);
 
 /* ---- helpers ------------------------------------------------------------------------ */
 /* Synchronises `stream`, copies the status word to the host and returns it (or

@@ -33,7 +33,7 @@ EXPORTS = [
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
     "antdt_weighted_aggregate_backup",
-    "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_read_status", "antdt_launch_count",
+    "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_read_status", "antdt_launch_count",
     "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_version",
 ]
 
@@ -128,6 +128,8 @@ def lib() -> C.CDLL:
         L.antdt_sparse_opt_update.argtypes = [P, I32, I64, I32, P, P, P, I64, I32, F, F, F, F, I64,
                                               P, P, P, P]
         L.antdt_bsp_step_host.argtypes = [P, P]
+        L.antdt_bsp_step_device.argtypes = [P, P]
+        L.antdt_bsp_step_device.restype = I32
         L.antdt_read_status.argtypes = [P, P]
         L.antdt_launch_count.restype = I64
         L.antdt_profile_enable.argtypes = [I32]
@@ -138,7 +140,7 @@ def lib() -> C.CDLL:
                    "antdt_dds_requeue_worker", "antdt_dds_counts", "antdt_dds_shard_info",
                    "antdt_dds_save", "antdt_dds_load", "antdt_ctl_create", "antdt_ctl_destroy",
     "antdt_ctl_report", "antdt_ctl_decide", "antdt_dd_solve", "antdt_embbag_fwd", "antdt_embbag_bwd_dedup",
-                   "antdt_weighted_aggregate", "antdt_sparse_opt_update", "antdt_bsp_step_host",
+                   "antdt_weighted_aggregate", "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device",
                    "antdt_read_status", "antdt_profile_enable", "antdt_profile_kernels",
                    "antdt_profile_get"):
             getattr(L, fn).restype = I32
@@ -386,6 +388,10 @@ def antdt_sparse_opt_update(table, ids, grads, n_ids_dev, opt: int, lr: float, e
 
 def antdt_bsp_step_host(desc: StepDesc, stream=None):
     _check(lib().antdt_bsp_step_host(C.byref(desc), _stream(stream)), "antdt_bsp_step_host")
+
+
+def antdt_bsp_step_device(desc: StepDesc, stream=None):
+    _check(lib().antdt_bsp_step_device(C.byref(desc), _stream(stream)), "antdt_bsp_step_device")
 
 
 def antdt_read_status(dev_status, stream=None) -> int:

@@ -114,3 +114,34 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
 #undef CK
   return ANTDT_OK;
 }
+
+// The same four calls for a batch that is already resident in device memory: nothing is copied,
+// no side stream is used, the status word is left as the caller set it.
+extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream) {
+  if (!d || d->nnz < 0 || d->n_bags < 0 || d->dim < 1 || !d->d_bag_offsets || !d->d_n_agg)
+    return ANTDT_ERR_INVALID_ARG;
+  const bool dense = d->d_dense_grads && d->dense_n > 0;
+  if (dense && !d->d_dense_out) return ANTDT_ERR_INVALID_ARG;
+  int32_t rc = antdt_embbag_fwd(d->table, d->dtype, d->n_rows, d->dim, d->d_row_ids, d->nnz,
+                                d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, stream);
+  if (rc != ANTDT_OK) return rc;
+  rc = antdt_embbag_bwd_dedup(d->d_row_ids, d->nnz, d->d_bag_offsets, d->n_bags, d->bags_per_sample,
+                              d->d_d_pooled, d->dim, d->n_rows, d->n_workers,
+                              d->worker_sample_offsets, d->d_uniq_ids, d->d_worker_uniq_offsets,
+                              d->d_seg_offsets, d->d_sorted_occ, d->d_uniq_grads, d->uniq_cap, d->ws,
+                              d->ws_bytes, d->d_status, stream);
+  if (rc != ANTDT_OK) return rc;
+  antdt_sparse_part sp;
+  sp.dim = d->dim; sp.n_rows = d->n_rows; sp.uniq_ids = d->d_uniq_ids;
+  sp.worker_uniq_offsets = d->d_worker_uniq_offsets; sp.uniq_grads = d->d_uniq_grads;
+  sp.in_cap = d->uniq_cap; sp.agg_ids = d->d_agg_ids; sp.agg_grads = d->d_agg_grads;
+  sp.n_agg = d->d_n_agg; sp.out_cap = d->agg_cap;
+  antdt_dense_part dp;
+  dp.grads = d->d_dense_grads; dp.n = d->dense_n; dp.stride = d->dense_n; dp.out = d->d_dense_out;
+  rc = antdt_weighted_aggregate(&sp, dense ? &dp : nullptr, d->batch_sizes, d->n_workers, d->ws,
+                                d->ws_bytes, d->d_status, stream);
+  if (rc != ANTDT_OK) return rc;
+  return antdt_sparse_opt_update(d->table, d->dtype, d->n_rows, d->dim, d->d_agg_ids, d->d_agg_grads,
+                                 d->d_n_agg, d->agg_cap, d->opt, d->lr, d->eps, d->beta1, d->beta2,
+                                 d->step, d->state0, d->state1, d->d_status, stream);
+}

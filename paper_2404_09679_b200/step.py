@@ -67,3 +67,45 @@ def run_step(buf: StepBuffers, table, state0, state1, oc: OptConfig, step: int, 
                                dense_out=buf.dense_out, dev_status=buf.status, stream=stream)
     B.antdt_sparse_opt_update(table, buf.agg_ids, buf.agg_grads, buf.n_agg, oc.opt, oc.lr, oc.eps,
                               oc.beta1, oc.beta2, step, state0, state1, buf.status, stream)
+
+
+class DeviceStep:
+    """One antdt_bsp_step_device call per step: the descriptor is filled once for a buffer set and
+    a model state, only the batch pointers and the step number change."""
+
+    def __init__(self, buf: StepBuffers, table, state0, state1, oc: OptConfig, n_workers: int):
+        import ctypes as C
+        self.buf, self.K = buf, n_workers
+        d = B.StepDesc()
+        p = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        d.table, d.dtype = p(table), (B.BF16 if table.dtype == torch.bfloat16 else B.F32)
+        d.n_rows, d.dim = table.shape
+        d.state0, d.state1 = p(state0), p(state1)
+        d.opt, d.lr, d.eps, d.beta1, d.beta2 = oc.opt, oc.lr, oc.eps, oc.beta1, oc.beta2
+        d.n_workers = n_workers
+        d.d_pooled_out, d.d_dense_out = p(buf.pooled), p(buf.dense_out)
+        d.d_uniq_ids, d.d_worker_uniq_offsets = p(buf.uniq_ids), p(buf.worker_uniq_offsets)
+        d.d_seg_offsets, d.d_sorted_occ = p(buf.seg_offsets), p(buf.sorted_occ)
+        d.d_uniq_grads, d.uniq_cap = p(buf.uniq_grads), buf.uniq_cap
+        d.d_agg_ids, d.d_agg_grads, d.d_n_agg, d.agg_cap = p(buf.agg_ids), p(buf.agg_grads), p(buf.n_agg), buf.agg_cap
+        d.ws, d.ws_bytes, d.d_status = p(buf.ws), buf.ws.numel(), p(buf.status)
+        self.desc = d
+        self._wso = (C.c_int64 * (n_workers + 1))()
+        self._bsz = (C.c_int64 * n_workers)()
+        d.worker_sample_offsets = C.cast(self._wso, C.c_void_p)
+        d.batch_sizes = C.cast(self._bsz, C.c_void_p)
+
+    def run(self, step: int, row_ids, bag_offsets, bags_per_sample: int, d_pooled,
+            worker_sample_offsets: Sequence[int], batch_sizes: Sequence[int], dense_grads=None,
+            stream=None):
+        d = self.desc
+        d.step = step
+        d.d_row_ids, d.nnz = row_ids.data_ptr(), row_ids.numel()
+        d.d_bag_offsets, d.n_bags = bag_offsets.data_ptr(), bag_offsets.numel() - 1
+        d.bags_per_sample = bags_per_sample
+        d.d_d_pooled = d_pooled.data_ptr()
+        d.d_dense_grads = None if dense_grads is None else dense_grads.data_ptr()
+        d.dense_n = 0 if dense_grads is None else dense_grads.shape[1]
+        self._wso[:] = [int(x) for x in worker_sample_offsets]
+        self._bsz[:] = [int(x) for x in batch_sizes]
+        B.antdt_bsp_step_device(d, stream)

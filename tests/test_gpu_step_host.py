@@ -91,3 +91,34 @@ def test_host_buffer_step_matches_device_calls_and_checker(cfg, scale):
             G.close(buf_b.agg_grads[:na].cpu().numpy(), want["agg"], rtol=3e-5, atol=2e-6)
         else:
             G.close_mostly(h_pooled.numpy(), want["pooled"], 1e-4, 1e-5, 1e-3, 2 * w.lr * w.len_hi)
+
+
+def test_single_call_device_step_equals_the_four_calls():
+    from paper_2404_09679_b200.step import DeviceStep
+    w = synth.WORKLOADS[3].scaled(B=1024, V=50_000, dense_n=8192)
+    plans = plan_steps(w, 2)
+    bm = synth.BatchMaker(w, "cuda")
+    table0 = bm.table()
+    oc = OptConfig(B.OPTS[w.opt], w.lr, w.eps, w.beta1, w.beta2)
+    t_a, t_b = table0.clone(), table0.clone()
+    z = lambda: torch.zeros(w.V, w.D, device="cuda")  # noqa: E731
+    s0_a, s1_a, s0_b, s1_b = z(), z(), z(), z()
+    buf_a = buf_b = ds = None
+    for s in range(2):
+        batch = make_batch(bm, plans[s], s)
+        nnz, n_bags = batch["row_ids"].numel(), batch["bag_offsets"].numel() - 1
+        if buf_a is None:
+            buf_a = StepBuffers(w.D, w.K, 2 * nnz, n_bags, w.dense_n)
+            buf_b = StepBuffers(w.D, w.K, 2 * nnz, n_bags, w.dense_n)
+            ds = DeviceStep(buf_b, t_b, s0_b, s1_b, oc, w.K)
+        args = (batch["row_ids"], batch["bag_offsets"], w.F, batch["d_pooled"], batch["wso"].tolist(),
+                batch["counts"].tolist(), batch["dense"])
+        run_step(buf_a, t_a, s0_a, s1_a, oc, s + 1, *args)
+        ds.run(s + 1, *args)
+        assert B.antdt_read_status(buf_a.status) == 0 and B.antdt_read_status(buf_b.status) == 0
+        na = int(buf_a.n_agg.item())
+        assert int(buf_b.n_agg.item()) == na
+        assert torch.equal(buf_b.pooled[:n_bags], buf_a.pooled[:n_bags])
+        assert torch.equal(buf_b.agg_grads[:na], buf_a.agg_grads[:na])
+        assert torch.equal(buf_b.dense_out, buf_a.dense_out)
+        assert torch.equal(t_b, t_a) and torch.equal(s0_b, s0_a) and torch.equal(s1_b, s1_a)
