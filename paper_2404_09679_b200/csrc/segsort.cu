@@ -496,6 +496,7 @@ SortLayout sort_layout(int S) {
   SortLayout L;
   const size_t C = (size_t)kSortChunksTarget + (size_t)S;
   L.max_chunks = (int)C;
+  L.n_segments = S;
   size_t o = 0;
   L.desc = o;        o = align_up(o + sizeof(SortDesc));
   L.seg_bounds = o;  o = align_up(o + 8 * ((size_t)S + 1));
@@ -546,7 +547,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
   int shift = 0;
   const uint32_t* kin = keys_in;
   const uint32_t* vin = vals_in;
-  const int S = L.max_chunks - kSortChunksTarget;
+  const int S = L.n_segments;
   for (int p = 0; p < P; ++p) {
     const int bits = (key_bits - shift + (P - p) - 1) / (P - p);
     const uint32_t mask = (1u << bits) - 1u;

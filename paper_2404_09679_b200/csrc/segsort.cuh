@@ -47,6 +47,7 @@ struct SortLayout {
   size_t chunk_runs;   // int64 [16 C + 1]  run counts per strip of a chunk (runs pass)
   size_t bytes;        // total
   int max_chunks;      // C
+  int n_segments;      // S
 };
 SortLayout sort_layout(int n_segments);
 
