@@ -17,10 +17,10 @@ pytestmark = pytest.mark.gpu
 
 CASES = {
     "c1": (synth.WORKLOADS[1], 10),
-    "c2": (synth.WORKLOADS[2].scaled(V=26 * 100_000), 6),
-    "c3": (synth.WORKLOADS[3].scaled(B=2048, V=200_000, dense_n=65_536), 3),
-    "c4": (synth.WORKLOADS[4].scaled(B=2048, V=1_000_000), 3),
-    "c5": (synth.WORKLOADS[5].scaled(B=16_384, V=500_000, dense_n=131_072), 3),
+    "c2": (synth.WORKLOADS[2].scaled(V=26 * 100_000), 10),
+    "c3": (synth.WORKLOADS[3].scaled(B=2048, V=200_000, dense_n=65_536), 5),
+    "c4": (synth.WORKLOADS[4].scaled(B=2048, V=1_000_000), 5),
+    "c5": (synth.WORKLOADS[5].scaled(B=16_384, V=500_000, dense_n=131_072), 5),
 }
 
 
