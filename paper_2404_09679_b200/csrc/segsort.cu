@@ -346,20 +346,20 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
 
 // ---------------------------------------------------------------------------------------
 // runs of equal keys
-// A chunk is cut into kRunStrips 32-aligned strips, one warp each.  count: heads per strip;
+// A chunk is cut into kRunStrips 128-aligned strips, one warp each.  count: heads per strip;
 // scan: exclusive scan over all strips of all chunks; emit: every warp walks its strip once,
-// knowing how many runs start before it.  No block barrier inside the walks; 8 x 32 keys are
-// loaded before the first is used.
+// knowing how many runs start before it.  A lane takes 4 consecutive keys (one 16-byte load), so
+// a warp step covers 128 keys = four whole words of the head-bit mask; two steps are in flight.
+// No block barrier inside the walks.
 // ---------------------------------------------------------------------------------------
 constexpr int kRunThreads = 512;
 constexpr int kRunStrips = kRunThreads / 32;  // 16
-constexpr int kRunUnroll = 8;
 
-struct Strip { int64_t s0, lo, hi; };  // aligned start, clipped [lo, hi)
+struct Strip { int64_t s0, lo, hi; };  // 128-aligned start, clipped [lo, hi)
 
 __device__ __forceinline__ Strip strip_of(int64_t b, int64_t e, int w) {
-  const int64_t ab = b & ~(int64_t)31;
-  const int64_t len = (((e - ab) + kRunStrips - 1) / kRunStrips + 31) & ~(int64_t)31;
+  const int64_t ab = b & ~(int64_t)127;
+  const int64_t len = (((e - ab) + kRunStrips - 1) / kRunStrips + 127) & ~(int64_t)127;
   Strip st;
   st.s0 = ab + (int64_t)w * len;
   st.lo = max(st.s0, b);
@@ -367,14 +367,41 @@ __device__ __forceinline__ Strip strip_of(int64_t b, int64_t e, int w) {
   return st;
 }
 
-// head flags of the 32 elements [i0, i0+32) of a strip; key = this lane's key (if in range)
-__device__ __forceinline__ bool head_at(const uint32_t* __restrict__ keys, int64_t i, const Strip& st,
-                                        int64_t seg_begin, uint32_t key, uint32_t prev_lane_key,
-                                        int lane) {
-  if (i < st.lo || i >= st.hi) return false;
-  if (i == seg_begin) return true;
-  const uint32_t prev = (lane == 0 || i == st.lo) ? __ldg(keys + i - 1) : prev_lane_key;
-  return key != prev;
+// The 4 keys [i, i+4) of a lane (i is a multiple of 4; the key buffers are 16-byte aligned).
+// Keys outside [lo, hi) are not loaded.
+__device__ __forceinline__ void load4(const uint32_t* __restrict__ keys, int64_t i, const Strip& st,
+                                      uint32_t (&k)[4]) {
+  if (i >= st.lo && i + 4 <= st.hi) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(keys + i));
+    k[0] = v.x; k[1] = v.y; k[2] = v.z; k[3] = v.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) k[j] = (i + j >= st.lo && i + j < st.hi) ? __ldg(keys + i + j) : 0u;
+  }
+}
+
+// 4-bit mask: bit j set iff key i+j is inside the strip and starts a run.  prev_k3 is the last
+// key of the lane to the left (meaningful when that key lies inside the strip).
+__device__ __forceinline__ unsigned heads4(const uint32_t* __restrict__ keys, int64_t i, const Strip& st,
+                                           int64_t seg_begin, const uint32_t (&k)[4], uint32_t prev_k3,
+                                           int lane) {
+  unsigned m = 0;
+  uint32_t prev = prev_k3;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int64_t e = i + j;
+    if (e >= st.lo && e < st.hi) {
+      bool h;
+      if (e == seg_begin) h = true;
+      else {
+        if (e == st.lo || (j == 0 && lane == 0)) prev = __ldg(keys + e - 1);
+        h = k[j] != prev;
+      }
+      m |= h ? (1u << j) : 0u;
+    }
+    prev = k[j];
+  }
+  return m;
 }
 
 __global__ void __launch_bounds__(kRunThreads)
@@ -388,19 +415,15 @@ runs_count_kernel(const uint32_t* __restrict__ keys, const SortDesc* __restrict_
   const Strip st = strip_of(chunk_begin[c], chunk_end[c], w);
   const int64_t seg_begin = seg_bounds[chunk_seg[c]];
   int cnt = 0;
-  for (int64_t j0 = st.s0; j0 < st.hi; j0 += 32 * kRunUnroll) {
-    uint32_t k[kRunUnroll];
-#pragma unroll
-    for (int r = 0; r < kRunUnroll; ++r) {
-      const int64_t i = j0 + r * 32 + lane;
-      k[r] = (i >= st.lo && i < st.hi) ? __ldg(keys + i) : 0u;
-    }
-#pragma unroll
-    for (int r = 0; r < kRunUnroll; ++r) {
-      const int64_t i = j0 + r * 32 + lane;
-      const uint32_t pk = __shfl_up_sync(0xffffffffu, k[r], 1);
-      cnt += head_at(keys, i, st, seg_begin, k[r], pk, lane) ? 1 : 0;
-    }
+  for (int64_t j0 = st.s0; j0 < st.hi; j0 += 256) {
+    uint32_t ka[4], kb[4];
+    const int64_t ia = j0 + lane * 4, ib = ia + 128;
+    load4(keys, ia, st, ka);
+    load4(keys, ib, st, kb);
+    const uint32_t pa = __shfl_up_sync(0xffffffffu, ka[3], 1);
+    const uint32_t pb = __shfl_up_sync(0xffffffffu, kb[3], 1);
+    cnt += __popc(heads4(keys, ia, st, seg_begin, ka, pa, lane));
+    cnt += __popc(heads4(keys, ib, st, seg_begin, kb, pb, lane));
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, o);
@@ -438,6 +461,53 @@ runs_scan_kernel(const SortDesc* __restrict__ desc, const int32_t* __restrict__ 
       seg_runs[s] = strip_runs[(size_t)seg_first[s] * kRunStrips];
 }
 
+// One warp step of the emit walk: the 128 keys [i0, i0+128), 4 per lane.
+__device__ __forceinline__ void emit_step(const uint32_t* __restrict__ keys, int64_t i0, const Strip& st,
+                                          int64_t b, int64_t e, int64_t seg_begin, const uint32_t (&k)[4],
+                                          int lane, int64_t& running, int32_t* __restrict__ uniq_keys,
+                                          int64_t* __restrict__ run_start, int64_t out_cap,
+                                          uint32_t* head_bits, int32_t* __restrict__ tile_first,
+                                          int tile_shift) {
+  const int64_t i = i0 + lane * 4;
+  const uint32_t prev = __shfl_up_sync(0xffffffffu, k[3], 1);
+  const unsigned m = heads4(keys, i, st, seg_begin, k, prev, lane);
+  // heads in the lanes to the left: inclusive warp scan of the per-lane counts
+  const int mine = __popc(m);
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  int64_t r = running + (incl - mine);  // runs that start before this lane's first key
+  if (tile_first && i >= st.lo && i < st.hi && (i & (((int64_t)1 << tile_shift) - 1)) == 0)
+    tile_first[i >> tile_shift] = (int32_t)(r + (m & 1u) - 1);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if ((m >> j) & 1u) {
+      if (r < out_cap) {
+        uniq_keys[r] = (int32_t)k[j];
+        run_start[r] = i + j;
+      }
+      ++r;
+    }
+  }
+  if (head_bits) {
+    // 8 lanes make one 32-bit word of the mask; words inside the chunk are stored whole, the
+    // chunk's first and last word (shared with a neighbour) are merged with an atomic OR
+    unsigned word = m << ((lane & 7) * 4);
+    word |= __shfl_xor_sync(0xffffffffu, word, 1);
+    word |= __shfl_xor_sync(0xffffffffu, word, 2);
+    word |= __shfl_xor_sync(0xffffffffu, word, 4);
+    if ((lane & 7) == 0 && word) {
+      const int64_t w0 = i0 + (lane >> 3) * 32;
+      if (w0 >= b && w0 + 32 <= e) head_bits[w0 >> 5] = word;
+      else atomicOr(&head_bits[w0 >> 5], word);
+    }
+  }
+  running += __shfl_sync(0xffffffffu, incl, 31);
+}
+
 __global__ void __launch_bounds__(kRunThreads)
 runs_emit_kernel(const uint32_t* __restrict__ keys, const SortDesc* __restrict__ desc,
                  const int32_t* __restrict__ chunk_seg, const int64_t* __restrict__ seg_bounds,
@@ -451,41 +521,16 @@ runs_emit_kernel(const uint32_t* __restrict__ keys, const SortDesc* __restrict__
   const int64_t b = chunk_begin[c], e = chunk_end[c];
   const Strip st = strip_of(b, e, w);
   const int64_t seg_begin = seg_bounds[chunk_seg[c]];
-  const int64_t tile_mask = ((int64_t)1 << tile_shift) - 1;
   int64_t running = strip_runs[(size_t)c * kRunStrips + w];  // runs that start before this strip
-  for (int64_t j0 = st.s0; j0 < st.hi; j0 += 32 * kRunUnroll) {
-    uint32_t k[kRunUnroll];
-#pragma unroll
-    for (int r = 0; r < kRunUnroll; ++r) {
-      const int64_t i = j0 + r * 32 + lane;
-      k[r] = (i >= st.lo && i < st.hi) ? __ldg(keys + i) : 0u;
-    }
-#pragma unroll
-    for (int r = 0; r < kRunUnroll; ++r) {
-      const int64_t i0 = j0 + r * 32;
-      if (i0 >= st.hi) break;
-      const int64_t i = i0 + lane;
-      const uint32_t pk = __shfl_up_sync(0xffffffffu, k[r], 1);
-      const bool head = head_at(keys, i, st, seg_begin, k[r], pk, lane);
-      const unsigned bal = __ballot_sync(0xffffffffu, head);
-      const int64_t incl = running + __popc(bal & ((2u << lane) - 1u));
-      if (head) {
-        const int64_t rr = incl - 1;
-        if (rr < out_cap) {
-          uniq_keys[rr] = (int32_t)k[r];
-          run_start[rr] = i;
-        }
-      }
-      if (tile_first && i >= st.lo && i < st.hi && (i & tile_mask) == 0)
-        tile_first[i >> tile_shift] = (int32_t)(incl - 1);
-      if (head_bits && lane == 0 && bal) {
-        // i0 is a multiple of 32: the ballot is exactly one word; words shared with another
-        // chunk (first / last word of the chunk) are merged with an atomic OR
-        if (i0 >= b && i0 + 32 <= e) head_bits[i0 >> 5] = bal;
-        else atomicOr(&head_bits[i0 >> 5], bal);
-      }
-      running += __popc(bal);
-    }
+  for (int64_t j0 = st.s0; j0 < st.hi; j0 += 256) {
+    uint32_t ka[4], kb[4];
+    load4(keys, j0 + lane * 4, st, ka);
+    load4(keys, j0 + 128 + lane * 4, st, kb);
+    emit_step(keys, j0, st, b, e, seg_begin, ka, lane, running, uniq_keys, run_start, out_cap,
+              head_bits, tile_first, tile_shift);
+    if (j0 + 128 < st.hi)
+      emit_step(keys, j0 + 128, st, b, e, seg_begin, kb, lane, running, uniq_keys, run_start, out_cap,
+                head_bits, tile_first, tile_shift);
   }
 }
 
