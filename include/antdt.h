@@ -355,6 +355,31 @@ int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream);
  * ignored, nothing is copied, and the status word is neither cleared nor read back.  One host
  * call instead of four: for small batches the per-call host cost is the step time. */
 int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream);
+/* The same device-resident step (Section II's iteration: local gradients, aggregation, update),
+ * replayed as ONE CUDA graph launch.  A step is 30-40 short kernels; on small batches their
+ * launches, not their run time, are the step time.  The first call with a given descriptor
+ * captures antdt_bsp_step_device on `stream` (thread-local capture mode), instantiates the graph
+ * and launches it; later calls whose descriptor is equal launch the kept executable graph.
+ *   - "Equal" covers every scalar and device pointer the device step reads, and the CONTENTS of
+ *     worker_sample_offsets[K+1] and batch_sizes[K] (they travel as kernel parameters); `step` is
+ *     compared only for Adam.  What the device pointers point at may differ from call to call.
+ *   - Up to 8 executable graphs are kept per device, least recently used replaced; a replaced
+ *     one is updated in place when the new capture has the same shape, else re-instantiated.  A
+ *     descriptor that changes every step therefore still runs as a graph, at the host cost of one
+ *     capture and update per step.
+ *   - Argument errors are those of the four calls, found while capturing; nothing runs then.
+ *   - If `stream` is already being captured by the caller, the four calls are issued into that
+ *     capture instead; a stream that cannot be captured (the legacy default stream) gets the
+ *     plain launches of antdt_bsp_step_device.
+ *   - Ownership: the graphs reference the caller's buffers; keep the buffers alive while graphs
+ *     that name them may be replayed, or drop the graphs with antdt_bsp_step_graph_reset.  The
+ *     executables are driver objects, the only thing this library ever creates on a device.
+ *   - Per-kernel event timing (antdt_profile_enable) does not see kernels inside a graph;
+ *     antdt_launch_count counts a replay's kernel nodes.
+ * Returns ANTDT_OK, an argument error, or ANTDT_ERR_CUDA. */
+int32_t antdt_bsp_step_graph(const antdt_step_desc* d, void* stream);
+/* Destroys the executable graphs kept for the current device. */
+int32_t antdt_bsp_step_graph_reset(void);
 
 /* ---- helpers ------------------------------------------------------------------------ */
 /* Synchronises `stream`, copies the status word to the host and returns it (or

@@ -33,7 +33,8 @@ EXPORTS = [
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
     "antdt_weighted_aggregate_backup",
-    "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_read_status", "antdt_launch_count",
+    "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_bsp_step_graph", "antdt_bsp_step_graph_reset",
+    "antdt_read_status", "antdt_launch_count",
     "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_version",
 ]
 
@@ -130,6 +131,10 @@ def lib() -> C.CDLL:
         L.antdt_bsp_step_host.argtypes = [P, P]
         L.antdt_bsp_step_device.argtypes = [P, P]
         L.antdt_bsp_step_device.restype = I32
+        L.antdt_bsp_step_graph.argtypes = [P, P]
+        L.antdt_bsp_step_graph.restype = I32
+        L.antdt_bsp_step_graph_reset.argtypes = []
+        L.antdt_bsp_step_graph_reset.restype = I32
         L.antdt_read_status.argtypes = [P, P]
         L.antdt_launch_count.restype = I64
         L.antdt_profile_enable.argtypes = [I32]
@@ -392,6 +397,14 @@ def antdt_bsp_step_host(desc: StepDesc, stream=None):
 
 def antdt_bsp_step_device(desc: StepDesc, stream=None):
     _check(lib().antdt_bsp_step_device(C.byref(desc), _stream(stream)), "antdt_bsp_step_device")
+
+
+def antdt_bsp_step_graph(desc: StepDesc, stream=None):
+    _check(lib().antdt_bsp_step_graph(C.byref(desc), _stream(stream)), "antdt_bsp_step_graph")
+
+
+def antdt_bsp_step_graph_reset():
+    _check(lib().antdt_bsp_step_graph_reset(), "antdt_bsp_step_graph_reset")
 
 
 def antdt_read_status(dev_status, stream=None) -> int:

@@ -12,6 +12,11 @@ namespace antdt {
 // ---- launch bookkeeping (runtime.cu) --------------------------------------------------
 int prof_begin(const char* name, cudaStream_t s);
 void prof_end(int token, cudaStream_t s);
+// While on, this thread's launches are counted but not bracketed by events (a stream that is
+// being captured cannot time its nodes).
+void prof_untimed(bool on);
+// Adds n to the launch counter: kernels that ran as nodes of a replayed graph.
+void count_launches(int64_t n);
 
 // Launch `kernel` and account for it (launch counter; CUDA-event bracket when profiling is on).
 #define ANTDT_LAUNCH(name, kernel, grid, block, smem, stream, ...)        \

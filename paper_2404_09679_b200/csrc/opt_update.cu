@@ -49,6 +49,10 @@ __device__ __forceinline__ float adam1(float& m, float& v, float g, float w, con
   return w - p.lr * (m / p.bc1) / (sqrtf(v / p.bc2) + p.eps);
 }
 
+// Rows a lane group has in flight.  Measured on B200: Adam (four 16-byte streams per row) gains
+// from two rows a stride apart; Adagrad is faster with one row and the higher occupancy.
+constexpr int kOptRowsAdam = 2;
+
 template <int G, int VPL, bool ADAM, bool BF16>
 __global__ void __launch_bounds__(kOptThreads)
 sparse_opt_kernel(void* table, int64_t n_rows, int dim, const int32_t* __restrict__ ids,
@@ -58,31 +62,46 @@ sparse_opt_kernel(void* table, int64_t n_rows, int dim, const int32_t* __restric
   const int nvec = dim / 4;
   const int64_t n = min(*n_ids_dev, max_ids);
   const int64_t stride = (int64_t)gridDim.x * (kOptThreads / G);
-  for (int64_t k = (int64_t)blockIdx.x * (kOptThreads / G) + threadIdx.x / G; k < n; k += stride) {
-    const int64_t row = ids[k];
-    if (row < 0 || row >= n_rows) {
-      if (lg == 0) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
-      continue;
+  constexpr int R = (ADAM && VPL == 1) ? kOptRowsAdam : 1;
+  for (int64_t k0 = (int64_t)blockIdx.x * (kOptThreads / G) + threadIdx.x / G; k0 < n; k0 += R * stride) {
+    int64_t row[R];
+    bool ok[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int64_t k = k0 + r * stride;
+      row[r] = k < n ? (int64_t)__ldg(ids + k) : -1;
+      ok[r] = row[r] >= 0 && row[r] < n_rows;
+      if (k < n && !ok[r] && lg == 0) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
     }
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int vi = lg + j * G;
       if (vi >= nvec) continue;
-      const size_t at = (size_t)row * dim + 4 * (size_t)vi;
-      const float4 g = ldg_f4(grads + (size_t)k * dim + 4 * vi);
-      float4 w = load_row4(table, BF16, at);
-      float4 s0 = *reinterpret_cast<const float4*>(state0 + at);
-      if (ADAM) {
-        float4 s1 = *reinterpret_cast<const float4*>(state1 + at);
-        w.x = adam1(s0.x, s1.x, g.x, w.x, p); w.y = adam1(s0.y, s1.y, g.y, w.y, p);
-        w.z = adam1(s0.z, s1.z, g.z, w.z, p); w.w = adam1(s0.w, s1.w, g.w, w.w, p);
-        *reinterpret_cast<float4*>(state1 + at) = s1;
-      } else {
-        w.x = adagrad1(s0.x, g.x, w.x, p); w.y = adagrad1(s0.y, g.y, w.y, p);
-        w.z = adagrad1(s0.z, g.z, w.z, p); w.w = adagrad1(s0.w, g.w, w.w, p);
+      float4 g[R], w[R], s0[R], s1[R];
+      size_t at[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (!ok[r]) continue;
+        at[r] = (size_t)row[r] * dim + 4 * (size_t)vi;
+        g[r] = ldg_f4(grads + (size_t)(k0 + r * stride) * dim + 4 * vi);
+        w[r] = load_row4(table, BF16, at[r]);
+        s0[r] = *reinterpret_cast<const float4*>(state0 + at[r]);
+        if (ADAM) s1[r] = *reinterpret_cast<const float4*>(state1 + at[r]);
       }
-      *reinterpret_cast<float4*>(state0 + at) = s0;
-      store_row4(table, BF16, at, w);
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (!ok[r]) continue;
+        if (ADAM) {
+          w[r].x = adam1(s0[r].x, s1[r].x, g[r].x, w[r].x, p); w[r].y = adam1(s0[r].y, s1[r].y, g[r].y, w[r].y, p);
+          w[r].z = adam1(s0[r].z, s1[r].z, g[r].z, w[r].z, p); w[r].w = adam1(s0[r].w, s1[r].w, g[r].w, w[r].w, p);
+          *reinterpret_cast<float4*>(state1 + at[r]) = s1[r];
+        } else {
+          w[r].x = adagrad1(s0[r].x, g[r].x, w[r].x, p); w[r].y = adagrad1(s0[r].y, g[r].y, w[r].y, p);
+          w[r].z = adagrad1(s0[r].z, g[r].z, w[r].z, p); w[r].w = adagrad1(s0[r].w, g[r].w, w[r].w, p);
+        }
+        *reinterpret_cast<float4*>(state0 + at[r]) = s0[r];
+        store_row4(table, BF16, at[r], w[r]);
+      }
     }
   }
 }

@@ -11,6 +11,7 @@ struct Pending { int slot; cudaEvent_t a, b; };
 
 std::mutex g_mu;
 bool g_profile = false;
+thread_local bool t_untimed = false;  // this thread is capturing a stream: no event brackets
 int64_t g_launches = 0;
 std::vector<Slot> g_slots;
 std::vector<Pending> g_pending;
@@ -67,7 +68,7 @@ void upload_small(const void* host, size_t bytes, void* dev, cudaStream_t s) {
 int prof_begin(const char* name, cudaStream_t s) {
   std::lock_guard<std::mutex> lk(g_mu);
   ++g_launches;
-  if (!g_profile) return -1;
+  if (!g_profile || t_untimed) return -1;
   int slot = -1;
   for (size_t i = 0; i < g_slots.size(); ++i)
     if (g_slots[i].name == name || strcmp(g_slots[i].name, name) == 0) { slot = (int)i; break; }
@@ -80,6 +81,13 @@ int prof_begin(const char* name, cudaStream_t s) {
   if (p.a) cudaEventRecord(p.a, s);
   g_pending.push_back(p);
   return (int)g_pending.size() - 1;
+}
+
+void prof_untimed(bool on) { t_untimed = on; }
+
+void count_launches(int64_t n) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  g_launches += n;
 }
 
 void prof_end(int token, cudaStream_t s) {

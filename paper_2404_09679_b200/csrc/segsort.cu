@@ -125,7 +125,9 @@ __device__ __forceinline__ void hist_add8(uint32_t* sh, const uint32_t (&k)[8], 
   atomicAdd(&sh[cur], cnt);
 }
 
-__global__ void __launch_bounds__(kSortThreads)
+constexpr int kHistThreads = 512;  // 3 CTAs per SM: all 48 warp slots hold loads in flight
+
+__global__ void __launch_bounds__(kHistThreads, kSortCtasPerSM)
 radix_hist_kernel(const uint32_t* __restrict__ keys, int shift, uint32_t mask,
                   const SortDesc* __restrict__ desc, const int64_t* __restrict__ chunk_begin,
                   const int64_t* __restrict__ chunk_end, uint32_t* __restrict__ hist,
@@ -134,7 +136,7 @@ radix_hist_kernel(const uint32_t* __restrict__ keys, int shift, uint32_t mask,
   if (c >= desc->n_chunks) return;
   __shared__ uint32_t sh[kSortMaxBins];
   const int tid = threadIdx.x;
-  for (int d = tid; d < kSortMaxBins; d += kSortThreads) sh[d] = 0;
+  for (int d = tid; d < kSortMaxBins; d += kHistThreads) sh[d] = 0;
   __syncthreads();
   const int64_t b = chunk_begin[c], e = chunk_end[c];
   const uint32_t limit = check_rows > 0 ? (uint32_t)check_rows : 0xffffffffu;
@@ -142,7 +144,7 @@ radix_hist_kernel(const uint32_t* __restrict__ keys, int shift, uint32_t mask,
   // groups of 8 keys that start on a 16-byte boundary, whatever the array's own alignment
   const int64_t off = (int64_t)((reinterpret_cast<uintptr_t>(keys) >> 2) & 3);
   const int64_t ab = ((b + off) & ~(int64_t)7) - off;
-  constexpr int64_t kStep = (int64_t)kSortThreads * 8;
+  constexpr int64_t kStep = (int64_t)kHistThreads * 8;
   for (int64_t base = ab + (int64_t)tid * 8; base < e; base += 2 * kStep) {
     const int64_t base2 = base + kStep;
     const bool full1 = base >= b && base + 8 <= e;
@@ -183,7 +185,7 @@ radix_hist_kernel(const uint32_t* __restrict__ keys, int shift, uint32_t mask,
   }
   if (kmax >= limit && check_rows > 0) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
   __syncthreads();
-  for (int d = tid; d < kSortMaxBins; d += kSortThreads) hist[(size_t)c * kSortMaxBins + d] = sh[d];
+  for (int d = tid; d < kSortMaxBins; d += kHistThreads) hist[(size_t)c * kSortMaxBins + d] = sh[d];
 }
 
 // ---------------------------------------------------------------------------------------
@@ -564,6 +566,21 @@ void segsort_setup(const int64_t* seg_bounds_dev, int S, int64_t n_cap, char* ws
                (int64_t*)(ws + L.chunk_begin), (int64_t*)(ws + L.chunk_end), L.max_chunks);
 }
 
+// Per device, once: opt in to the scatter's 55 KB of dynamic shared memory (3 CTAs per SM).
+// Not a stream operation; callers that capture a stream call it before the capture starts.
+void segsort_prepare_device() {
+  static bool attr_set[64] = {};
+  int dev_id = 0;
+  cudaGetDevice(&dev_id);
+  bool& done = attr_set[dev_id & 63];
+  if (done) return;
+  cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       (int)kScatSmem);
+  cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                       cudaSharedmemCarveoutMaxShared);
+  done = true;
+}
+
 void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* keys_out,
                  uint32_t* vals_out, uint32_t* keys_tmp, uint32_t* vals_tmp, int key_bits,
                  int64_t check_rows, char* ws, const SortLayout& L, int32_t* status,
@@ -577,17 +594,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
   uint32_t* hist = (uint32_t*)(ws + L.hist);
   uint32_t* bin_base = (uint32_t*)(ws + L.bin_base);
   const int P = sort_passes(key_bits);
-  static bool attr_set[64] = {};
-  int dev_id = 0;
-  cudaGetDevice(&dev_id);
-  bool& carveout_set = attr_set[dev_id & 63];
-  if (!carveout_set) {  // per device: opt in to 55 KB of dynamic shared memory, 3 CTAs per SM
-    cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         (int)kScatSmem);
-    cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                         cudaSharedmemCarveoutMaxShared);
-    carveout_set = true;
-  }
+  segsort_prepare_device();
   // spread the bits evenly over the passes
   int shift = 0;
   const uint32_t* kin = keys_in;
@@ -600,7 +607,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
     const bool to_out = ((P - 1 - p) % 2) == 0;
     uint32_t* kout = to_out ? keys_out : keys_tmp;
     uint32_t* vout = to_out ? vals_out : vals_tmp;
-    ANTDT_LAUNCH(agg ? "agg_radix_hist" : "radix_hist", radix_hist_kernel, L.max_chunks, kSortThreads, 0, s, kin, shift,
+    ANTDT_LAUNCH(agg ? "agg_radix_hist" : "radix_hist", radix_hist_kernel, L.max_chunks, kHistThreads, 0, s, kin, shift,
                  mask, desc, chunk_begin, chunk_end, hist, p == 0 ? check_rows : (int64_t)0, status);
     ANTDT_LAUNCH(agg ? "agg_radix_scan" : "radix_scan", radix_scan_kernel, S, kSortMaxBins, 0, s, desc, seg_first, hist,
                  bin_base);

@@ -60,6 +60,9 @@ inline int bits_for(int64_t n_values) {  // bits needed for values in [0, n_valu
   return b;
 }
 
+// Sets the kernel attributes the sort needs on the current device (idempotent, cheap).
+void segsort_prepare_device();
+
 // seg_bounds_dev: int64 [S+1] device, ascending, last = element count (<= n_cap).  Builds the
 // chunk descriptors in `ws` (laid out by sort_layout).
 void segsort_setup(const int64_t* seg_bounds_dev, int n_segments, int64_t n_cap, char* ws,

@@ -1,7 +1,11 @@
 // One whole BSP step from host buffers: stage in, run the four device calls, stage out.
+#include <string.h>
+
 #include <mutex>
+#include <vector>
 
 #include "common.cuh"
+#include "segsort.cuh"
 
 namespace {
 // Side streams and events of the host-buffer step, created on first use for each device.
@@ -144,4 +148,147 @@ extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream)
   return antdt_sparse_opt_update(d->table, d->dtype, d->n_rows, d->dim, d->d_agg_ids, d->d_agg_grads,
                                  d->d_n_agg, d->agg_cap, d->opt, d->lr, d->eps, d->beta1, d->beta2,
                                  d->step, d->state0, d->state1, d->d_status, stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// The device-resident step replayed as a CUDA graph.
+// A step is 30-40 short launches; on small batches the launches, not the kernels, are the step
+// time.  The four calls are captured once per distinct descriptor and replayed with a single
+// graph launch.  Everything a captured launch depends on is in the key: every scalar and device
+// pointer of the descriptor and the CONTENTS of the two host arrays (they reach the device as
+// kernel parameters).  What the pointers point at may change freely between replays.
+// ---------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kGraphSlots = 8;  // executable graphs kept per device
+
+struct GraphEntry {
+  std::vector<uint64_t> key;
+  cudaGraphExec_t exec = nullptr;
+  int64_t n_kernels = 0;
+  uint64_t tick = 0;
+};
+struct GraphCache {
+  std::vector<GraphEntry> entries;
+  uint64_t tick = 0;
+};
+GraphCache g_gc[64];
+std::mutex g_gc_mu;
+
+uint64_t bits_of(const void* p) { return (uint64_t)reinterpret_cast<uintptr_t>(p); }
+uint64_t bits_of(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+
+std::vector<uint64_t> graph_key(const antdt_step_desc* d) {
+  std::vector<uint64_t> k;
+  const int K = d->n_workers;
+  k.reserve(48 + 2 * (size_t)K);
+  const bool adam = d->opt == ANTDT_OPT_ADAM;
+  const uint64_t head[] = {
+      bits_of(d->table), (uint64_t)d->dtype, (uint64_t)d->n_rows, (uint64_t)d->dim,
+      bits_of(d->state0), bits_of(d->state1), (uint64_t)d->opt, bits_of(d->lr), bits_of(d->eps),
+      bits_of(d->beta1), bits_of(d->beta2),
+      adam ? (uint64_t)d->step : (uint64_t)(d->step >= 1),  // Adagrad does not use the step number
+      (uint64_t)d->nnz, (uint64_t)d->n_bags, (uint64_t)d->bags_per_sample, (uint64_t)d->dense_n,
+      (uint64_t)K, bits_of(d->d_row_ids), bits_of(d->d_bag_offsets), bits_of(d->d_pooled_out),
+      bits_of(d->d_d_pooled), bits_of(d->d_dense_grads), bits_of(d->d_dense_out),
+      bits_of(d->d_uniq_ids), bits_of(d->d_worker_uniq_offsets), bits_of(d->d_seg_offsets),
+      bits_of(d->d_sorted_occ), bits_of(d->d_uniq_grads), (uint64_t)d->uniq_cap,
+      bits_of(d->d_agg_ids), bits_of(d->d_agg_grads), bits_of(d->d_n_agg), (uint64_t)d->agg_cap,
+      bits_of(d->ws), (uint64_t)d->ws_bytes, bits_of(d->d_status)};
+  k.assign(head, head + sizeof(head) / sizeof(head[0]));
+  for (int i = 0; i <= K; ++i) k.push_back((uint64_t)d->worker_sample_offsets[i]);
+  for (int i = 0; i < K; ++i) k.push_back((uint64_t)d->batch_sizes[i]);
+  return k;
+}
+}  // namespace
+
+extern "C" int32_t antdt_bsp_step_graph(const antdt_step_desc* d, void* stream) {
+  if (!d || d->n_workers < 1 || d->n_workers > antdt::kMaxSegments || !d->worker_sample_offsets ||
+      !d->batch_sizes)
+    return ANTDT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cs) != cudaSuccess) {
+    cudaGetLastError();
+    return ANTDT_ERR_CUDA;
+  }
+  // inside somebody else's capture the launches simply join that graph
+  if (cs != cudaStreamCaptureStatusNone) return antdt_bsp_step_device(d, stream);
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ANTDT_ERR_CUDA;
+  const std::vector<uint64_t> key = graph_key(d);
+
+  std::lock_guard<std::mutex> lk(g_gc_mu);
+  GraphCache& gc = g_gc[dev];
+  ++gc.tick;
+  for (GraphEntry& e : gc.entries) {
+    if (e.key == key) {
+      e.tick = gc.tick;
+      if (cudaGraphLaunch(e.exec, s) != cudaSuccess) return ANTDT_ERR_CUDA;
+      antdt::count_launches(e.n_kernels);
+      return ANTDT_OK;
+    }
+  }
+
+  // miss: capture the four calls
+  antdt::segsort_prepare_device();
+  if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();  // e.g. the legacy default stream cannot be captured: plain launches
+    return antdt_bsp_step_device(d, stream);
+  }
+  const int64_t before = antdt_launch_count();
+  antdt::prof_untimed(true);
+  const int32_t rc = antdt_bsp_step_device(d, stream);
+  antdt::prof_untimed(false);
+  const int64_t n_kernels = antdt_launch_count() - before;
+  antdt::count_launches(-n_kernels);  // captured, not run
+  cudaGraph_t g = nullptr;
+  const cudaError_t ce = cudaStreamEndCapture(s, &g);
+  if (rc != ANTDT_OK || ce != cudaSuccess || !g) {
+    if (g) cudaGraphDestroy(g);
+    cudaGetLastError();
+    return rc != ANTDT_OK ? rc : ANTDT_ERR_CUDA;
+  }
+
+  GraphEntry* slot = nullptr;
+  if (gc.entries.size() < kGraphSlots) {
+    gc.entries.emplace_back();
+    slot = &gc.entries.back();
+  } else {  // least recently used; its executable is updated in place when the shape matches
+    slot = &gc.entries[0];
+    for (GraphEntry& e : gc.entries)
+      if (e.tick < slot->tick) slot = &e;
+  }
+  if (slot->exec) {
+    cudaGraphExecUpdateResultInfo info;
+    if (cudaGraphExecUpdate(slot->exec, g, &info) != cudaSuccess) {
+      cudaGetLastError();
+      cudaGraphExecDestroy(slot->exec);
+      slot->exec = nullptr;
+    }
+  }
+  if (!slot->exec && cudaGraphInstantiate(&slot->exec, g, 0) != cudaSuccess) {
+    cudaGetLastError();
+    cudaGraphDestroy(g);
+    slot->exec = nullptr;
+    slot->key.clear();
+    slot->tick = 0;
+    return ANTDT_ERR_CUDA;
+  }
+  cudaGraphDestroy(g);
+  slot->key = key;
+  slot->n_kernels = n_kernels;
+  slot->tick = gc.tick;
+  if (cudaGraphLaunch(slot->exec, s) != cudaSuccess) return ANTDT_ERR_CUDA;
+  antdt::count_launches(n_kernels);
+  return ANTDT_OK;
+}
+
+extern "C" int32_t antdt_bsp_step_graph_reset(void) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ANTDT_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_gc_mu);
+  for (GraphEntry& e : g_gc[dev].entries)
+    if (e.exec) cudaGraphExecDestroy(e.exec);
+  g_gc[dev].entries.clear();
+  return ANTDT_OK;
 }

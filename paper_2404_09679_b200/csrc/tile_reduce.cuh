@@ -196,25 +196,49 @@ tile_fixup_kernel(const TileArgs a) {
   if (o_end >= n) return;  // the last tile's runs all end inside it
   const int dim = a.dim;
   const int nvec = dim / 4;
-  uint32_t hb[kRedTile / 32 + 1];
+  // The pass is a chain of dependent loads for little data, so everything whose address only
+  // depends on the tile index is requested up front: the head bits of this tile and the next
+  // (a straddling run nearly always ends there), the run index, this tile's tail piece and the
+  // next tile's head piece.  (The mask and the partial arrays reach one tile past the end.)
+  constexpr int kW = kRedTile / 32;
+  uint32_t hb[2 * kW + 1];
 #pragma unroll
-  for (int i = 0; i <= kRedTile / 32; ++i) hb[i] = __ldg(a.head_bits + (o_begin >> 5) + i);
-  if (hb[kRedTile / 32] & 1u) return;  // next tile starts a new run: nothing straddles
-  int heads = 0;
-#pragma unroll
-  for (int i = 0; i < kRedTile / 32; ++i) heads += __popc(hb[i]);
-  if (heads == 0) return;  // the straddling run started earlier: its start tile owns it
-  const int64_t u = (int64_t)a.tile_first[tile] + heads - ((hb[0] & 1u) ? 1 : 0);
-  if (u >= a.out_cap) return;
-
-  float4 tot[VPL];
+  for (int i = 0; i <= 2 * kW; ++i) hb[i] = __ldg(a.head_bits + (o_begin >> 5) + i);
+  const int32_t first_run = __ldg(a.tile_first + tile);
+  float4 tot[VPL], nxt[VPL];
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
     const int vi = lg + k * G;
-    tot[k] = vi < nvec ? reinterpret_cast<const float4*>(a.tail_part + (size_t)tile * dim)[vi]
-                       : make_float4(0.f, 0.f, 0.f, 0.f);
+    const bool in = vi < nvec;
+    tot[k] = in ? reinterpret_cast<const float4*>(a.tail_part + (size_t)tile * dim)[vi]
+                : make_float4(0.f, 0.f, 0.f, 0.f);
+    nxt[k] = in ? reinterpret_cast<const float4*>(a.head_part + (size_t)(tile + 1) * dim)[vi]
+                : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  for (int64_t t2 = tile + 1;; ++t2) {
+  float scale = 1.f;
+  if (!AGG) {  // worker of the run = worker of any of its entries (searched while the loads fly)
+    int w = interval_of(a.bounds, a.K + 1, o_end - 1);
+    if (w > a.K - 1) w = a.K - 1;
+    scale = a.scales[w];
+  }
+  if (hb[kW] & 1u) return;  // next tile starts a new run: nothing straddles
+  int heads = 0;
+#pragma unroll
+  for (int i = 0; i < kW; ++i) heads += __popc(hb[i]);
+  if (heads == 0) return;  // the straddling run started earlier: its start tile owns it
+  const int64_t u = (int64_t)first_run + heads - ((hb[0] & 1u) ? 1 : 0);
+  if (u >= a.out_cap) return;
+
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    tot[k].x += nxt[k].x; tot[k].y += nxt[k].y; tot[k].z += nxt[k].z; tot[k].w += nxt[k].w;
+  }
+  // does the run go on past tile+1?  (no head inside it nor at the start of the tile after it)
+  bool open = o_end + kRedTile < n;
+#pragma unroll
+  for (int i = kW; i < 2 * kW; ++i) open = open && hb[i] == 0u;
+  open = open && (hb[2 * kW] & 1u) == 0u;
+  for (int64_t t2 = tile + 2; open; ++t2) {
     const int64_t b2 = t2 * kRedTile;
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
@@ -226,15 +250,9 @@ tile_fixup_kernel(const TileArgs a) {
     if (b2 + kRedTile >= n) break;  // ran to the end of the array
     bool ends = false;              // a head inside t2, or at the start of the tile after it
 #pragma unroll
-    for (int i = 0; i < kRedTile / 32; ++i) ends |= __ldg(a.head_bits + (b2 >> 5) + i) != 0u;
-    ends |= (__ldg(a.head_bits + (b2 >> 5) + kRedTile / 32) & 1u) != 0u;
+    for (int i = 0; i < kW; ++i) ends |= __ldg(a.head_bits + (b2 >> 5) + i) != 0u;
+    ends |= (__ldg(a.head_bits + (b2 >> 5) + kW) & 1u) != 0u;
     if (ends) break;
-  }
-  float scale = 1.f;
-  if (!AGG) {  // worker of the run = worker of any of its entries
-    int w = interval_of(a.bounds, a.K + 1, o_end - 1);
-    if (w > a.K - 1) w = a.K - 1;
-    scale = a.scales[w];
   }
   float* dst = a.out + (size_t)u * dim;
 #pragma unroll

@@ -97,7 +97,8 @@ class DeviceStep:
 
     def run(self, step: int, row_ids, bag_offsets, bags_per_sample: int, d_pooled,
             worker_sample_offsets: Sequence[int], batch_sizes: Sequence[int], dense_grads=None,
-            stream=None):
+            stream=None, graph: bool = False):
+        """graph=True replays the step as one CUDA graph launch (antdt_bsp_step_graph)."""
         d = self.desc
         d.step = step
         d.d_row_ids, d.nnz = row_ids.data_ptr(), row_ids.numel()
@@ -108,4 +109,7 @@ class DeviceStep:
         d.dense_n = 0 if dense_grads is None else dense_grads.shape[1]
         self._wso[:] = [int(x) for x in worker_sample_offsets]
         self._bsz[:] = [int(x) for x in batch_sizes]
-        B.antdt_bsp_step_device(d, stream)
+        if graph:
+            B.antdt_bsp_step_graph(d, stream)
+        else:
+            B.antdt_bsp_step_device(d, stream)
