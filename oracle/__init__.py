@@ -43,6 +43,10 @@ _lib.orc_aggregate_sparse.argtypes = [C.c_int, _p, _p, _p, _p, C.c_int, _p, _p, 
 _lib.orc_aggregate_dense.argtypes = [_p, C.c_int64, C.c_int64, _p, C.c_int, _p]
 _lib.orc_sparse_opt_update.argtypes = [_p, C.c_int, C.c_int64, C.c_int, _p, _p, C.c_int64, C.c_int,
                                        C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64, _p, _p]
+_lib.orc_sparse_rowwise_adagrad.argtypes = [_p, C.c_int, C.c_int64, C.c_int, _p, _p, C.c_int64,
+                                            C.c_float, C.c_float, _p]
+_lib.orc_dense_opt_update.argtypes = [_p, _p, C.c_int64, C.c_int, C.c_float, C.c_float, C.c_float,
+                                      C.c_float, C.c_int64, _p, _p]
 
 _lib.orc_ctl_decide.argtypes = [_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_double, _p, _p, _p, _p]
 
@@ -191,6 +195,29 @@ def sparse_opt_update(table, ids, grads, opt, lr, eps, beta1, beta2, step, state
                                     ids.shape[0], OPTS[opt], lr, eps, beta1, beta2, step,
                                     _ptr(_chk(state0, _f32)),
                                     _ptr(None if state1 is None else _chk(state1, _f32)))
+    if rc:
+        raise OracleError(rc)
+
+
+def sparse_rowwise_adagrad(table, ids, grads, lr, eps, state0):
+    """In place on table and state0 (numpy [n_rows] float32: one accumulator per row)."""
+    t, dt = _table_view(table)
+    V, D = t.shape
+    assert state0.shape == (V,)
+    rc = _lib.orc_sparse_rowwise_adagrad(_ptr(t), dt, V, D, _ptr(_chk(ids, _i32)),
+                                         _ptr(_chk(grads, _f32)), ids.shape[0], lr, eps,
+                                         _ptr(_chk(state0, _f32)))
+    if rc:
+        raise OracleError(rc)
+
+
+def dense_opt_update(params, grad, opt, lr, eps, beta1, beta2, step, state0, state1=None):
+    """In place on params / state0 / state1 (numpy float32 vectors of one length)."""
+    n = params.shape[0]
+    assert grad.shape == (n,) and state0.shape == (n,)
+    rc = _lib.orc_dense_opt_update(_ptr(_chk(params, _f32)), _ptr(_chk(grad, _f32)), n, OPTS[opt],
+                                   lr, eps, beta1, beta2, step, _ptr(_chk(state0, _f32)),
+                                   _ptr(None if state1 is None else _chk(state1, _f32)))
     if rc:
         raise OracleError(rc)
 

@@ -444,6 +444,55 @@ int orc_sparse_opt_update(void* table, int dtype, i64 n_rows, int dim, const i32
   return OK;
 }
 
+// Row-wise Adagrad: ONE accumulator per row, fed with the mean of the row's squared gradient
+// elements:  acc_r += (1/D) sum_c g_c^2;  w_c -= lr * g_c / (sqrt(acc_r) + eps).
+// s0 is [n_rows].  (The servers' update, Section II, with the accumulator shared by a row.)
+int orc_sparse_rowwise_adagrad(void* table, int dtype, i64 n_rows, int dim, const i32* ids,
+                               const float* grads, i64 n_ids, float lr, float eps, float* s0) {
+  for (i64 k = 0; k < n_ids; ++k)
+    if (ids[k] < 0 || ids[k] >= n_rows) return E_ID;
+  for (i64 k = 0; k < n_ids; ++k) {
+    double sq = 0.0;
+    for (int c = 0; c < dim; ++c) {
+      double g = (double)grads[k * dim + c];
+      sq += g * g;
+    }
+    double acc = (double)s0[ids[k]] + sq / (double)dim;
+    s0[ids[k]] = (float)acc;
+    for (int c = 0; c < dim; ++c) {
+      i64 at = (i64)ids[k] * dim + c;
+      double w = load_elem(table, dtype, at);
+      w -= (double)lr * (double)grads[k * dim + c] / (std::sqrt(acc) + (double)eps);
+      store_elem(table, dtype, at, w);
+    }
+  }
+  return OK;
+}
+
+// Optimizer step on a dense fp32 parameter vector with the aggregated dense gradient (Section
+// II: the servers update the parameters after aggregating): the same element-wise Adagrad /
+// Adam formulas as the sparse update, every element touched.
+int orc_dense_opt_update(float* w, const float* grad, i64 n, int opt, float lr, float eps, float b1,
+                         float b2, i64 t, float* s0, float* s1) {
+  double c1 = 1.0 - std::pow((double)b1, (double)t), c2 = 1.0 - std::pow((double)b2, (double)t);
+  for (i64 e = 0; e < n; ++e) {
+    double g = (double)grad[e], x = (double)w[e];
+    if (opt == 0) {
+      double acc = (double)s0[e] + g * g;
+      s0[e] = (float)acc;
+      x -= (double)lr * g / (std::sqrt(acc) + (double)eps);
+    } else {
+      double m = (double)b1 * (double)s0[e] + (1.0 - (double)b1) * g;
+      double v = (double)b2 * (double)s1[e] + (1.0 - (double)b2) * g * g;
+      s0[e] = (float)m;
+      s1[e] = (float)v;
+      x -= (double)lr * (m / c1) / (std::sqrt(v / c2) + (double)eps);
+    }
+    w[e] = (float)x;
+  }
+  return OK;
+}
+
 // AntDT-ND controller, worker side (Section VI-A steps 2-5), stateless form: the whole report
 // history is passed in.  reports: n_rep rows (worker, batch size, BPT seconds) in arrival order.
 // Window means over each worker's last Lt / Lp reports; straggler if mean_i >= lambda * mean over

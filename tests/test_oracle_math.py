@@ -256,6 +256,91 @@ def test_update_rejects_out_of_range_id():
                                  "adagrad", 0.01, 1e-8, 0, 0, 1, np.zeros((3, 4), np.float32))
 
 
+# ---- row-wise Adagrad and the dense update -------------------------------------------------
+def test_rowwise_adagrad_closed_form_constant_gradient():
+    V, D, T = 5, 4, 6
+    lr, eps = 0.05, 1e-8
+    W = np.full((V, D), -0.25, np.float32)
+    acc = np.zeros(V, np.float32)
+    g = np.array([[0.25, -0.5, 1.0, 2.0]], np.float32)
+    ids = np.array([2], np.int32)
+    for _ in range(T):
+        oracle.sparse_rowwise_adagrad(W, ids, g, lr, eps, acc)
+    g64 = g[0].astype(np.float64)
+    ms = (g64 ** 2).sum() / D                      # the row's mean square: 5.3125 / 4
+    assert ms == 1.328125
+    assert np.allclose(acc[2], T * ms, rtol=1e-6)
+    want = -0.25 - np.float64(np.float32(lr)) * sum(
+        g64 / (np.sqrt(t * ms) + np.float64(np.float32(eps))) for t in range(1, T + 1))
+    assert np.allclose(W[2], want, rtol=1e-6)
+    mask = np.arange(V) != 2
+    assert np.all(W[mask] == np.float32(-0.25)) and np.all(acc[mask] == 0)
+
+
+def test_rowwise_adagrad_equals_elementwise_when_magnitudes_are_equal():
+    # |g_c| = c for every element: the row's mean square is c^2, which is what every element's
+    # own accumulator holds, so the two variants move the row identically (closed form of the
+    # element-wise rule: acc = t c^2)
+    lr, eps, c = 0.01, 1e-8, 0.75
+    g = np.array([[c, -c, -c, c, c, -c, c, c]], np.float32)
+    W = np.zeros((2, 8), np.float32)
+    acc = np.zeros(2, np.float32)
+    ids = np.array([1], np.int32)
+    for _ in range(3):
+        oracle.sparse_rowwise_adagrad(W, ids, g, lr, eps, acc)
+    lr64, eps64 = np.float64(np.float32(lr)), np.float64(np.float32(eps))
+    want = -lr64 * np.sign(g[0]) * sum(c / (np.sqrt(t) * c + eps64) for t in (1, 2, 3))
+    assert np.allclose(W[1], want, rtol=1e-6)
+    assert np.isclose(acc[1], 3 * c * c, rtol=1e-6)
+    # dim 1: the row IS the element, so the stored state equals the element-wise call's
+    W1, W2 = np.full((3, 1), 0.5, np.float32), np.full((3, 1), 0.5, np.float32)
+    a1, a2 = np.zeros(3, np.float32), np.zeros((3, 1), np.float32)
+    g1 = np.array([[0.3], [-2.0]], np.float32)
+    i1 = np.array([0, 2], np.int32)
+    for t in (1, 2):
+        oracle.sparse_rowwise_adagrad(W1, i1, g1, lr, eps, a1)
+        oracle.sparse_opt_update(W2, i1, g1, "adagrad", lr, eps, 0, 0, t, a2)
+    assert np.array_equal(W1, W2) and np.array_equal(a1, a2[:, 0])
+
+
+def test_rowwise_adagrad_zero_gradient_and_bad_id():
+    W = np.full((3, 4), 0.3, np.float32)
+    acc = np.full(3, 2.0, np.float32)
+    oracle.sparse_rowwise_adagrad(W, np.array([1], np.int32), np.zeros((1, 4), np.float32), 0.01,
+                                  1e-8, acc)
+    assert np.all(W == np.float32(0.3)) and np.all(acc == 2.0)
+    with pytest.raises(oracle.OracleError):
+        oracle.sparse_rowwise_adagrad(W, np.array([3], np.int32), np.zeros((1, 4), np.float32),
+                                      0.01, 1e-8, acc)
+
+
+def test_dense_update_closed_forms():
+    lr, eps, b1, b2 = 1e-2, 1e-8, 0.9, 0.999
+    g = np.array([0.5, -0.25, 3.0, -1e-3, 0.0], np.float32)
+    g64 = g.astype(np.float64)
+    lr64, eps64 = np.float64(np.float32(lr)), np.float64(np.float32(eps))
+    # Adagrad, constant gradient: acc_T = T g^2, w_T = w_0 - lr sum_t g / (sqrt(t)|g| + eps)
+    w = np.full(5, 1.0, np.float32)
+    acc = np.zeros(5, np.float32)
+    for t in range(1, 5):
+        oracle.dense_opt_update(w, g, "adagrad", lr, eps, 0, 0, t, acc)
+    assert np.allclose(acc, 4 * g64 ** 2, rtol=1e-6)
+    want = 1.0 - lr64 * sum(g64 / (np.sqrt(t) * np.abs(g64) + eps64) for t in range(1, 5))
+    assert np.allclose(w, want, rtol=1e-6)
+    assert w[4] == 1.0 and acc[4] == 0.0            # zero gradient: element untouched
+    # Adam, constant gradient: every step moves -lr g / (|g| + eps)
+    w = np.zeros(5, np.float32)
+    m = np.zeros(5, np.float32)
+    v = np.zeros(5, np.float32)
+    step = -lr64 * g64 / (np.abs(g64) + eps64)
+    for t in range(1, 5):
+        oracle.dense_opt_update(w, g, "adam", lr, eps, b1, b2, t, m, v)
+        assert np.allclose(w, t * step, rtol=2e-6, atol=1e-10)
+    b1d, b2d = np.float64(np.float32(b1)), np.float64(np.float32(b2))
+    assert np.allclose(m, (1 - b1d ** 4) * g64, rtol=1e-6)
+    assert np.allclose(v, (1 - b2d ** 4) * g64 ** 2, rtol=1e-6)
+
+
 # ---- backup-workers aggregation --------------------------------------------------------------
 def test_backup_aggregate_is_the_mean_over_the_surviving_samples():
     rng = np.random.default_rng(40)
