@@ -65,7 +65,7 @@ enum {
 
 enum { ANTDT_F32 = 0, ANTDT_BF16 = 1 };                  /* table row element type        */
 enum { ANTDT_RULE_PROPORTIONAL = 0, ANTDT_RULE_MINMAX = 1 };
-enum { ANTDT_OPT_ADAGRAD = 0, ANTDT_OPT_ADAM = 1 };
+enum { ANTDT_OPT_ADAGRAD = 0, ANTDT_OPT_ADAM = 1, ANTDT_OPT_ROWWISE_ADAGRAD = 2 };
 enum { ANTDT_SHARD_TODO = 0, ANTDT_SHARD_DOING = 1, ANTDT_SHARD_DONE = 2 };
 
 /* ===================================================================================== */
@@ -304,6 +304,9 @@ int32_t antdt_weighted_aggregate_backup(const antdt_sparse_part* sp, const antdt
  *   Adagrad: state0 += g*g;  w -= lr * g / (sqrt(state0) + eps)
  *   Adam:    state0 = b1*state0 + (1-b1)*g;  state1 = b2*state1 + (1-b2)*g*g;
  *            w -= lr * (state0/(1-b1^step)) / (sqrt(state1/(1-b2^step)) + eps)
+ *   Row-wise Adagrad (one accumulator per ROW, for tables whose optimizer state must stay a
+ *            1/dim fraction of the table):  state0[row] += (1/dim) sum_c g_c*g_c;
+ *            w_c -= lr * g_c / (sqrt(state0[row]) + eps);  state0 is device [n_rows] fp32.
  * step is the global 1-based iteration.  Arithmetic is fp32; bf16 rows are widened, updated
  * and stored back round-to-nearest-even.  ids must be distinct (aggregate's output is).
  *   table  device [n_rows, dim] dtype, in/out      state0/state1 device [n_rows, dim] fp32
@@ -314,6 +317,16 @@ int32_t antdt_sparse_opt_update(void* table, int32_t dtype, int64_t n_rows, int3
                                 const int64_t* n_ids_dev, int64_t max_ids, int32_t opt, float lr,
                                 float eps, float beta1, float beta2, int64_t step, float* state0,
                                 float* state1, int32_t* dev_status, void* stream);
+
+/* Server update of the DENSE parameters (Section II: after aggregating, the servers update
+ * the parameters): the element-wise Adagrad / Adam formulas above on a dense fp32 vector, with
+ * the gradient antdt_weighted_aggregate's dense part produced.  Every element is touched.
+ *   params, state0, state1 (Adam only): device [n] fp32, in/out      grad: device [n] fp32
+ *   n % 4 == 0, all pointers 16-byte aligned; opt is ANTDT_OPT_ADAGRAD or ANTDT_OPT_ADAM.
+ * Asynchronous on stream; returns ANTDT_OK, ANTDT_ERR_INVALID_ARG or ANTDT_ERR_CUDA. */
+int32_t antdt_dense_opt_update(float* params, const float* grad, int64_t n, int32_t opt, float lr,
+                               float eps, float beta1, float beta2, int64_t step, float* state0,
+                               float* state1, void* stream);
 
 /* One whole step from HOST buffers: copies the step's inputs to the caller's device staging
  * buffers, runs fwd, bwd_dedup, aggregate and update in order on `stream`, and copies the

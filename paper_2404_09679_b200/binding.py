@@ -16,10 +16,10 @@ OK, ERR_INVALID_ARG, ERR_ID_OUT_OF_RANGE, ERR_WORKSPACE_TOO_SMALL, ERR_CAPACITY,
     ERR_TIMEOUT, ERR_EXHAUSTED, ERR_STATE, ERR_BAD_OFFSETS, ERR_INFEASIBLE = range(11)
 F32, BF16 = 0, 1
 RULE_PROPORTIONAL, RULE_MINMAX = 0, 1
-OPT_ADAGRAD, OPT_ADAM = 0, 1
+OPT_ADAGRAD, OPT_ADAM, OPT_ROWWISE_ADAGRAD = 0, 1, 2
 SHARD_TODO, SHARD_DOING, SHARD_DONE = 0, 1, 2
 RULES = {"proportional": RULE_PROPORTIONAL, "minmax": RULE_MINMAX}
-OPTS = {"adagrad": OPT_ADAGRAD, "adam": OPT_ADAM}
+OPTS = {"adagrad": OPT_ADAGRAD, "adam": OPT_ADAM, "rowwise_adagrad": OPT_ROWWISE_ADAGRAD}
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libantdt.so")
 _lib = None
@@ -33,7 +33,7 @@ EXPORTS = [
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
     "antdt_weighted_aggregate_backup",
-    "antdt_sparse_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_bsp_step_graph", "antdt_bsp_step_graph_reset",
+    "antdt_sparse_opt_update", "antdt_dense_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_bsp_step_graph", "antdt_bsp_step_graph_reset",
     "antdt_read_status", "antdt_launch_count",
     "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_version",
 ]
@@ -128,6 +128,8 @@ def lib() -> C.CDLL:
         L.antdt_weighted_aggregate_backup.restype = I32
         L.antdt_sparse_opt_update.argtypes = [P, I32, I64, I32, P, P, P, I64, I32, F, F, F, F, I64,
                                               P, P, P, P]
+        L.antdt_dense_opt_update.argtypes = [P, P, I64, I32, F, F, F, F, I64, P, P, P]
+        L.antdt_dense_opt_update.restype = I32
         L.antdt_bsp_step_host.argtypes = [P, P]
         L.antdt_bsp_step_device.argtypes = [P, P]
         L.antdt_bsp_step_device.restype = I32
@@ -389,6 +391,13 @@ def antdt_sparse_opt_update(table, ids, grads, n_ids_dev, opt: int, lr: float, e
         _dp(table), _dtype_code(table), V, D, _dp(ids), _dp(grads), _dp(n_ids_dev), ids.numel(),
         opt, lr, eps, beta1, beta2, step, _dp(state0), _dp(state1), _dp(dev_status),
         _stream(stream)), "antdt_sparse_opt_update")
+
+
+def antdt_dense_opt_update(params, grad, opt: int, lr: float, eps: float, beta1: float,
+                           beta2: float, step: int, state0, state1=None, stream=None):
+    _check(lib().antdt_dense_opt_update(_dp(params), _dp(grad), params.numel(), opt, lr, eps, beta1,
+                                        beta2, step, _dp(state0), _dp(state1), _stream(stream)),
+           "antdt_dense_opt_update")
 
 
 def antdt_bsp_step_host(desc: StepDesc, stream=None):

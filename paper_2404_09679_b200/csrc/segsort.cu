@@ -281,11 +281,19 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
     }
     __syncthreads();  // (A) also: the previous tile's write-out is over
 
+    // peer masks of all items first (independent, their latencies overlap), counters after
+    unsigned pm[kScatItems];
 #pragma unroll
     for (int i = 0; i < kScatItems; ++i) {
       const bool valid = wbase + i * 32 < tile_n;
       const uint32_t d = valid ? ((k[i] >> shift) & mask) : (uint32_t)kSortMaxBins;
-      const unsigned m = __match_any_sync(0xffffffffu, d);
+      pm[i] = __match_any_sync(0xffffffffu, d);
+    }
+#pragma unroll
+    for (int i = 0; i < kScatItems; ++i) {
+      const bool valid = wbase + i * 32 < tile_n;
+      const uint32_t d = (k[i] >> shift) & mask;
+      const unsigned m = pm[i];
       // every peer reads the counter (one broadcast), the first peer then bumps it
       const uint32_t old = valid ? my_wh[d] : 0u;
       __syncwarp();

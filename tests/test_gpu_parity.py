@@ -287,6 +287,70 @@ def test_update_textbook_cases_and_flags():
     assert np.all(gw[[0, 3]] == 1.0) and np.all(gw[[1, 2]] == 0.5) and np.all(acc[[1, 2]] == 1.0)
 
 
+@pytest.mark.parametrize("D,bf16", [(4, False), (16, False), (64, False), (200, False), (64, True), (8, True)])
+def test_rowwise_adagrad_matches_checker(D, bf16):
+    rng = np.random.default_rng(100 + D)
+    V, n = 3000, 1100
+    W = rng.normal(0, 0.01, size=(V, D)).astype(np.float32)
+    Wt = _bf16_bits(W) if bf16 else W
+    acc = np.abs(rng.normal(0, 0.1, size=V)).astype(np.float32)
+    ids = np.sort(rng.choice(V, size=n, replace=False)).astype(np.int32)
+    g = rng.normal(0, 0.05, size=(n, D)).astype(np.float32)
+    gw, g0, _, code = G.gpu_update(Wt, ids, g, "rowwise_adagrad", 0.01, 1e-8, 0.0, 0.0, 2, acc)
+    assert code == 0
+    w_ref, r0 = Wt.copy(), acc.copy()
+    oracle.sparse_rowwise_adagrad(w_ref, ids, g, 0.01, 1e-8, r0)
+    G.close(g0, r0)
+    if bf16:
+        a = (gw.astype(np.uint32) << 16).view(np.float32)
+        b = (w_ref.astype(np.uint32) << 16).view(np.float32)
+        G.close(a, b, rtol=G.BF16_RTOL, atol=1e-6)
+        assert (gw != w_ref).mean() < 0.02
+    else:
+        G.close(gw, w_ref)
+    untouched = np.ones(V, bool)
+    untouched[ids] = False
+    assert np.array_equal(gw[untouched], Wt[untouched]) and np.array_equal(g0[untouched], acc[untouched])
+    # out-of-range id: flagged and skipped, the other rows still updated
+    W1 = np.ones((4, 8), np.float32)
+    gw, a1, _, code = G.gpu_update(W1, np.array([1, 9, 2], np.int32), np.ones((3, 8), np.float32),
+                                   "rowwise_adagrad", 0.5, 0.0, 0, 0, 1, np.zeros(4, np.float32))
+    assert code == B.ERR_ID_OUT_OF_RANGE
+    assert np.all(gw[[0, 3]] == 1.0) and np.all(gw[[1, 2]] == 0.5) and a1.tolist() == [0, 1, 1, 0]
+
+
+@pytest.mark.parametrize("opt", ["adagrad", "adam"])
+@pytest.mark.parametrize("n", [4, 1000, 1 << 20, (1 << 22) + 12])
+def test_dense_update_matches_checker(opt, n):
+    rng = np.random.default_rng(n % 1000 + (opt == "adam"))
+    w = rng.normal(0, 0.1, size=n).astype(np.float32)
+    g = rng.normal(0, 0.01, size=n).astype(np.float32)
+    s0 = np.abs(rng.normal(0, 0.1, size=n)).astype(np.float32)
+    s1 = np.abs(rng.normal(0, 0.01, size=n)).astype(np.float32) if opt == "adam" else None
+    lr, eps, b1, b2, step = (0.01, 1e-8, 0.0, 0.0, 3) if opt == "adagrad" else (1e-3, 1e-8, 0.9, 0.999, 5)
+    dw, dg, d0 = G.dev(w), G.dev(g), G.dev(s0)
+    d1 = None if s1 is None else G.dev(s1)
+    B.antdt_dense_opt_update(dw, dg, B.OPTS[opt], lr, eps, b1, b2, step, d0, d1)
+    torch.cuda.synchronize()
+    oracle.dense_opt_update(w, g, opt, lr, eps, b1, b2, step, s0, s1)
+    G.close(dw.cpu().numpy(), w)
+    G.close(d0.cpu().numpy(), s0)
+    if s1 is not None:
+        G.close(d1.cpu().numpy(), s1)
+
+
+def test_dense_update_argument_errors_and_empty():
+    z = torch.zeros(8, device="cuda")
+    B.antdt_dense_opt_update(z[:0], z[:0], B.OPT_ADAGRAD, 0.1, 1e-8, 0, 0, 1, z[:0])   # n = 0: nothing
+    for bad in (lambda: B.antdt_dense_opt_update(z[:6], z[:6], B.OPT_ADAGRAD, 0.1, 1e-8, 0, 0, 1, z[:6]),
+                lambda: B.antdt_dense_opt_update(z, z.clone(), B.OPT_ADAM, 0.1, 1e-8, .9, .99, 1, z.clone()),
+                lambda: B.antdt_dense_opt_update(z, z.clone(), B.OPT_ROWWISE_ADAGRAD, 0.1, 1e-8, 0, 0, 1, z.clone()),
+                lambda: B.antdt_dense_opt_update(z, z.clone(), B.OPT_ADAGRAD, 0.1, 1e-8, 0, 0, 0, z.clone())):
+        with pytest.raises(B.AntdtError) as ei:
+            bad()
+        assert ei.value.code == B.ERR_INVALID_ARG
+
+
 # ---- limits of the worker count, and the parts of the aggregate on their own ------------------
 def test_a_thousand_workers():
     rng = np.random.default_rng(41)
