@@ -1,12 +1,14 @@
 // Server aggregation: batch-size weighted sum of the workers' mean gradients.
 //
-// Sparse part: the workers' row lists (each ascending) are merged by one stable radix sort of
+// Sparse part, up to 32 workers: the range-partitioned merge of agg_range.cu (no sort).
+// Sparse part, more workers: the workers' row lists (each ascending) are merged by one stable radix sort of
 // (row id, position in the concatenated list); equal rows then sit together in ascending
 // worker order, and the tile-parallel segmented reduction (tile_reduce.cuh) forms each row's
 // weighted sum of its <= K contributions in that fixed order.  Because the sorted positions of
 // one worker ascend with the row id, the gather of the workers' gradient rows is K
 // forward-moving streams, not a random walk.
 // Dense part: a K-way streaming reduction, one 16-byte vector per thread and worker.
+#include "agg_range.cuh"
 #include "segsort.cuh"
 #include "tile_reduce.cuh"
 
@@ -17,6 +19,8 @@ size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct AggLayout {
   SortLayout sort;
+  RangeLayout range;
+  size_t range_ws;
   size_t sort_ws, bounds, weights, wuo, cwuo, drop, keys_a, keys_b, src, vals_t, run_start, head_bits,
       tile_first, head_part, tail_part, bytes;
 };
@@ -42,6 +46,11 @@ AggLayout agg_layout(int64_t in_cap, int K, int dim) {
   L.tile_first = o; o = align_up(o + 4 * (n_tiles + 1));
   L.head_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
   L.tail_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
+  L.range_ws = o;
+  if (K <= kRangeMaxWorkers) {  // scratch of the range-partitioned merge (up to 32 workers)
+    L.range = range_layout(K);
+    o = align_up(o + L.range.bytes);
+  }
   L.bytes = o;
   return L;
 }
@@ -166,6 +175,50 @@ extern "C" size_t antdt_weighted_aggregate_workspace_bytes(int64_t in_cap, int32
 
 namespace antdt {
 namespace {
+// More than 32 workers: merge order by one stable radix sort of (row id, position).
+void sort_merge_order(const antdt_sparse_part* sp, const uint8_t* dropped, bool any_dropped, int K,
+                      int64_t in_cap, int64_t agg_cap, char* w8, const AggLayout& L,
+                      int32_t* dev_status, cudaStream_t s) {
+    char* sort_ws = w8 + L.sort_ws;
+    int64_t* bounds = (int64_t*)(w8 + L.bounds);
+    uint32_t* keys_a = (uint32_t*)(w8 + L.keys_a);
+    const uint32_t* sort_keys = reinterpret_cast<const uint32_t*>(sp->uniq_ids);
+    const uint32_t* sort_vals = nullptr;  // payload = position in the concatenated lists
+    const int key_bits = bits_for(sp->n_rows);
+    if (!any_dropped) {
+      ANTDT_LAUNCH("agg_prep", agg_prep_kernel, 1, 256, 0, s, sp->worker_uniq_offsets, K, in_cap,
+                   bounds, (int64_t*)(w8 + L.wuo), dev_status);
+    } else {
+      uint32_t hd[kMaxSegments];
+      for (int i = 0; i < K; ++i) hd[i] = dropped[i] ? 1u : 0u;
+      uint32_t* d_drop = (uint32_t*)(w8 + L.drop);
+      int64_t* cwuo = (int64_t*)(w8 + L.cwuo);
+      upload_small(hd, 4 * (size_t)K, d_drop, s);
+      ANTDT_LAUNCH("agg_prep", agg_prep_backup_kernel, 1, 32, 0, s, sp->worker_uniq_offsets, d_drop,
+                   K, in_cap, bounds, (int64_t*)(w8 + L.wuo), cwuo, dev_status);
+      // the compacted input lives in the pair of sort buffers that the first pass does not
+      // write: the temporaries when the pass count is odd, the outputs when it is even
+      const bool odd = sort_passes(key_bits) % 2 == 1;
+      uint32_t* keys_c = (uint32_t*)(w8 + (odd ? L.keys_b : L.keys_a));
+      uint32_t* vals_c = (uint32_t*)(w8 + (odd ? L.vals_t : L.src));
+      if (in_cap > 0) {
+        int64_t want = (in_cap + 255) / 256;
+        const int64_t gcap = (int64_t)kNumSM * 16;
+        ANTDT_LAUNCH("agg_compact", agg_compact_kernel, (unsigned)(want > gcap ? gcap : want), 256,
+                     16 * ((size_t)K + 1) + 4 * (size_t)K, s, sp->uniq_ids,
+                     (const int64_t*)(w8 + L.wuo), cwuo, d_drop, K, keys_c, vals_c);
+      }
+      sort_keys = keys_c;
+      sort_vals = vals_c;
+    }
+    segsort_setup(bounds, 1, in_cap, sort_ws, L.sort, s);
+    segsort_run(sort_keys, sort_vals, keys_a, (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b),
+                (uint32_t*)(w8 + L.vals_t), key_bits, 0, sort_ws, L.sort, dev_status, s, true);
+    segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
+                 agg_cap, (uint32_t*)(w8 + L.head_bits),
+                 (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s, true);
+}
+
 int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
                        const int64_t* batch_sizes, const uint8_t* dropped, int32_t n_workers,
                        void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
@@ -207,44 +260,20 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
   upload_small(hw, 4 * (size_t)K, w8 + L.weights, s);
 
   if (sp) {
-    char* sort_ws = w8 + L.sort_ws;
     int64_t* bounds = (int64_t*)(w8 + L.bounds);
-    uint32_t* keys_a = (uint32_t*)(w8 + L.keys_a);
-    const uint32_t* sort_keys = reinterpret_cast<const uint32_t*>(sp->uniq_ids);
-    const uint32_t* sort_vals = nullptr;  // payload = position in the concatenated lists
-    const int key_bits = bits_for(sp->n_rows);
-    if (!any_dropped) {
-      ANTDT_LAUNCH("agg_prep", agg_prep_kernel, 1, 256, 0, s, sp->worker_uniq_offsets, K, in_cap,
-                   bounds, (int64_t*)(w8 + L.wuo), dev_status);
+    const int64_t agg_cap = sp->out_cap < in_cap ? sp->out_cap : in_cap;
+    if (K <= kRangeMaxWorkers && in_cap > 0) {
+      // up to 32 workers: the merge order comes from the range-partitioned pass, no sort
+      uint32_t dropped_bits = 0;
+      for (int i = 0; i < K; ++i)
+        if (dropped && dropped[i]) dropped_bits |= 1u << i;
+      range_merge_order(sp->uniq_ids, sp->worker_uniq_offsets, in_cap, sp->n_rows, K, dropped_bits,
+                        sp->agg_ids, sp->n_agg, agg_cap, (int64_t*)(w8 + L.wuo), bounds,
+                        (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.head_bits),
+                        (int32_t*)(w8 + L.tile_first), kRedTile, w8 + L.range_ws, L.range, dev_status, s);
     } else {
-      uint32_t hd[kMaxSegments];
-      for (int i = 0; i < K; ++i) hd[i] = dropped[i] ? 1u : 0u;
-      uint32_t* d_drop = (uint32_t*)(w8 + L.drop);
-      int64_t* cwuo = (int64_t*)(w8 + L.cwuo);
-      upload_small(hd, 4 * (size_t)K, d_drop, s);
-      ANTDT_LAUNCH("agg_prep", agg_prep_backup_kernel, 1, 32, 0, s, sp->worker_uniq_offsets, d_drop,
-                   K, in_cap, bounds, (int64_t*)(w8 + L.wuo), cwuo, dev_status);
-      // the compacted input lives in the pair of sort buffers that the first pass does not
-      // write: the temporaries when the pass count is odd, the outputs when it is even
-      const bool odd = sort_passes(key_bits) % 2 == 1;
-      uint32_t* keys_c = (uint32_t*)(w8 + (odd ? L.keys_b : L.keys_a));
-      uint32_t* vals_c = (uint32_t*)(w8 + (odd ? L.vals_t : L.src));
-      if (in_cap > 0) {
-        int64_t want = (in_cap + 255) / 256;
-        const int64_t gcap = (int64_t)kNumSM * 16;
-        ANTDT_LAUNCH("agg_compact", agg_compact_kernel, (unsigned)(want > gcap ? gcap : want), 256,
-                     16 * ((size_t)K + 1) + 4 * (size_t)K, s, sp->uniq_ids,
-                     (const int64_t*)(w8 + L.wuo), cwuo, d_drop, K, keys_c, vals_c);
-      }
-      sort_keys = keys_c;
-      sort_vals = vals_c;
+      sort_merge_order(sp, dropped, any_dropped, K, in_cap, agg_cap, w8, L, dev_status, s);
     }
-    segsort_setup(bounds, 1, in_cap, sort_ws, L.sort, s);
-    segsort_run(sort_keys, sort_vals, keys_a, (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b),
-                (uint32_t*)(w8 + L.vals_t), key_bits, 0, sort_ws, L.sort, dev_status, s, true);
-    segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
-                 sp->out_cap < in_cap ? sp->out_cap : in_cap, (uint32_t*)(w8 + L.head_bits),
-                 (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s, true);
     if (in_cap > 0) {
       TileArgs t;
       t.payload = (const uint32_t*)(w8 + L.src);

@@ -4,6 +4,7 @@
 #include <mutex>
 #include <vector>
 
+#include "agg_range.cuh"
 #include "common.cuh"
 #include "segsort.cuh"
 
@@ -231,6 +232,7 @@ extern "C" int32_t antdt_bsp_step_graph(const antdt_step_desc* d, void* stream) 
 
   // miss: capture the four calls
   antdt::segsort_prepare_device();
+  antdt::range_prepare_device();
   if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();  // e.g. the legacy default stream cannot be captured: plain launches
     return antdt_bsp_step_device(d, stream);
