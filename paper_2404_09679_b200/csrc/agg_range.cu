@@ -113,20 +113,18 @@ __device__ __forceinline__ void entry_of(int e, const int32_t* s_beg, const int3
   j = s_beg[lo] + (e - s_off[lo]);
 }
 
-// mask[kl] = set of workers whose list holds row id (b << r_log2) + kl.  Two barriers.
-__device__ __forceinline__ void range_build_mask(uint32_t* mask, int R, const int32_t* __restrict__ ids,
-                                                 int entries, int64_t b, int r_log2, int64_t n_rows,
-                                                 const int32_t* s_beg, const int32_t* s_off,
-                                                 int32_t* status) {
-  uint4* m4 = reinterpret_cast<uint4*>(mask);
-  for (int i = threadIdx.x; i < R / 4; i += kRaThreads) m4[i] = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  const uint32_t base_key = (uint32_t)(b << r_log2);
+// One pass over the range's entries, a batch of loads in flight per thread.  f(w, j, id, kl)
+// for the entries whose row id lies in the range and in the table; the others raise
+// ID_OUT_OF_RANGE and are skipped.
+template <typename F>
+__device__ __forceinline__ void for_each_entry(const int32_t* __restrict__ ids, int entries, int R,
+                                               uint32_t base_key, int64_t n_rows, const int32_t* s_beg,
+                                               const int32_t* s_off, int32_t* status, F f) {
   for (int e0 = threadIdx.x; e0 < entries; e0 += kRaBatch * kRaThreads) {
     int w[kRaBatch], j[kRaBatch];
     uint32_t id[kRaBatch];
 #pragma unroll
-    for (int t = 0; t < kRaBatch; ++t) {  // the batch's loads are in flight together
+    for (int t = 0; t < kRaBatch; ++t) {
       const int e = e0 + t * kRaThreads;
       entry_of(e < entries ? e : e0, s_beg, s_off, w[t], j[t]);
       id[t] = (uint32_t)__ldg(ids + j[t]);
@@ -135,43 +133,60 @@ __device__ __forceinline__ void range_build_mask(uint32_t* mask, int R, const in
     for (int t = 0; t < kRaBatch; ++t) {
       if (e0 + t * kRaThreads >= entries) break;
       const uint32_t kl = id[t] - base_key;
-      if (kl < (uint32_t)R && (int64_t)id[t] < n_rows) atomicOr(&mask[kl], 1u << w[t]);
-      else set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);  // skipped: not part of the union
+      if (kl < (uint32_t)R && (int64_t)id[t] < n_rows) f(w[t], j[t], id[t], kl);
+      else set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
     }
   }
+}
+
+// Exclusive prefix sums of two per-thread counts over the CTA's 256 threads; totals returned
+// through the references.  s_tmp: 16 ints.  Two barriers.
+__device__ __forceinline__ void block_scan2(int& a, int& b, int& tot_a, int& tot_b, int32_t* s_tmp) {
+  const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+  int ia = a, ib = b;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int ta = __shfl_up_sync(0xffffffffu, ia, o), tb = __shfl_up_sync(0xffffffffu, ib, o);
+    if (lane >= o) { ia += ta; ib += tb; }
+  }
+  if (lane == 31) { s_tmp[wp] = ia; s_tmp[kRaWarps + wp] = ib; }
+  __syncthreads();
+  int pa = 0, pb = 0;
+  tot_a = 0; tot_b = 0;
+#pragma unroll
+  for (int i = 0; i < kRaWarps; ++i) {
+    const int va = s_tmp[i], vb = s_tmp[kRaWarps + i];
+    pa += i < wp ? va : 0; pb += i < wp ? vb : 0;
+    tot_a += va; tot_b += vb;
+  }
+  a = pa + ia - a;
+  b = pb + ib - b;
   __syncthreads();
 }
 
+// Distinct row ids of range b: one presence bit per row id of the range.
 __global__ void __launch_bounds__(kRaThreads)
 range_count_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ bnd,
                    const int64_t* __restrict__ wuo, int K, int64_t P, int r_log2, int64_t n_rows,
                    uint32_t dropped, int32_t* __restrict__ distinct, int32_t* status) {
-  extern __shared__ __align__(16) unsigned char ra_smem[];
+  __shared__ uint32_t pres[(1 << kRangeMaxLog2) / 32];
+  __shared__ int64_t s_before;
+  __shared__ int32_t s_beg[32], s_off[33], s_tmp[2 * kRaWarps];
   const int R = 1 << r_log2;
-  uint32_t* mask = reinterpret_cast<uint32_t*>(ra_smem);
-  int64_t* s_before = reinterpret_cast<int64_t*>(mask + R);
-  int32_t* s_beg = reinterpret_cast<int32_t*>(s_before + 1);
-  int32_t* s_off = s_beg + 32;   // [33]
-  int32_t* s_cnt = s_off + 33;   // [8] warp counts
   const int64_t b = blockIdx.x;
-  const Pieces pc = range_pieces(bnd, wuo, K, P, b, dropped, s_beg, s_off, s_before);
+  const Pieces pc = range_pieces(bnd, wuo, K, P, b, dropped, s_beg, s_off, &s_before);
   if (pc.entries == 0) {
     if (threadIdx.x == 0) distinct[b] = 0;
     return;
   }
-  range_build_mask(mask, R, ids, pc.entries, b, r_log2, n_rows, s_beg, s_off, status);
-  const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
-  const int per = R / kRaWarps;
-  int cnt = 0;
-  for (int i = 0; i < per; i += 32) cnt += __popc(__ballot_sync(0xffffffffu, mask[wp * per + i + lane] != 0u));
-  if (lane == 0) s_cnt[wp] = cnt;
+  if (threadIdx.x < R / 32) pres[threadIdx.x] = 0u;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int d = 0;
-#pragma unroll
-    for (int i = 0; i < kRaWarps; ++i) d += s_cnt[i];
-    distinct[b] = d;
-  }
+  for_each_entry(ids, pc.entries, R, (uint32_t)(b << r_log2), n_rows, s_beg, s_off, status,
+                 [&](int, int, uint32_t, uint32_t kl) { atomicOr(&pres[kl >> 5], 1u << (kl & 31)); });
+  __syncthreads();
+  int cnt = threadIdx.x < R / 32 ? __popc(pres[threadIdx.x]) : 0, zero = 0, tot, tz;
+  block_scan2(cnt, zero, tot, tz, s_tmp);
+  if (threadIdx.x == 0) distinct[b] = tot;
 }
 
 // Exclusive scan of distinct[P] -> base[P+1]; one CTA of 1024 threads, consecutive ranges per
@@ -221,6 +236,10 @@ range_scan_kernel(const int32_t* __restrict__ distinct, int64_t P, int64_t* __re
 // a head bit where a row's contributions start, agg_ids, and the run index of every entry whose
 // slot starts a reduction tile.  slot = entries of earlier ranges + contributions of smaller row
 // ids of this range + earlier workers holding the same row id.
+//
+// Shared memory: mask[R] (worker set per row id), pres[R/32] (presence bits: the table is
+// sparse, so everything after the fill walks presence words and present ids only), per presence
+// word the present ids before it (wrank), per present id the contributions before it (first_c).
 __global__ void __launch_bounds__(kRaThreads)
 range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ bnd,
                   const int64_t* __restrict__ wuo, int K, int64_t P, int r_log2, int64_t n_rows,
@@ -229,15 +248,18 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
                   int32_t* __restrict__ tile_first, int tile_shift, int32_t* status) {
   extern __shared__ __align__(16) unsigned char ra_smem[];
   const int R = 1 << r_log2;
+  const int nW = R / 32;  // presence words: at most 256 = one per thread
   uint32_t* mask = reinterpret_cast<uint32_t*>(ra_smem);
-  uint32_t* info = mask + R;  // per present local id: rank | contributions before it << 13
-  int64_t* s_before = reinterpret_cast<int64_t*>(info + R);
-  int32_t* s_beg = reinterpret_cast<int32_t*>(s_before + 1);
+  uint32_t* first_c = mask + R;
+  int64_t* s_before = reinterpret_cast<int64_t*>(first_c + R);
+  uint32_t* pres = reinterpret_cast<uint32_t*>(s_before + 1);  // [256]
+  int32_t* wrank = reinterpret_cast<int32_t*>(pres + 256);     // [256]
+  int32_t* s_beg = wrank + 256;  // [32]
   int32_t* s_off = s_beg + 32;   // [33]
-  int32_t* s_cnt = s_off + 33;   // [8] distinct per warp, [8] contributions per warp
-  uint32_t* hb = reinterpret_cast<uint32_t*>(s_cnt + 16);  // head bits of this range's slots
+  int32_t* s_tmp = s_off + 33;   // [16]
+  uint32_t* hb = reinterpret_cast<uint32_t*>(s_tmp + 16);  // head bits of this range's slots
   const int64_t b = blockIdx.x;
-  const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+  const int tid = threadIdx.x;
   const int64_t u0 = __ldg(base + b);  // requested now: every global round trip here is serial
   const Pieces pc = range_pieces(bnd, wuo, K, P, b, dropped, s_beg, s_off, s_before);
   if (pc.entries == 0) return;
@@ -245,46 +267,34 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   const int hb_shift = (int)(pc.before & 31);
   const int n_hw = (hb_shift + pc.entries + 31) >> 5;
   for (int i = tid; i < n_hw; i += kRaThreads) hb[i] = 0u;
-  range_build_mask(mask, R, ids, pc.entries, b, r_log2, n_rows, s_beg, s_off, status);
-
-  // two exclusive prefix sums over the table in id order: present words, set bits.  Warp w owns
-  // words [w*R/8, (w+1)*R/8); a lane reads word start + i*32 + lane.
-  const int per = R / kRaWarps;
-  const unsigned lt = (1u << lane) - 1u;
-  int n_pres = 0, n_bits = 0;
-  for (int i = 0; i < per; i += 32) {
-    const uint32_t m = mask[wp * per + i + lane];
-    n_pres += __popc(__ballot_sync(0xffffffffu, m != 0u));
-    n_bits += __popc(m);
+  if (tid < nW) pres[tid] = 0u;
+  {
+    uint4* m4 = reinterpret_cast<uint4*>(mask);
+    for (int i = tid; i < R / 4; i += kRaThreads) m4[i] = make_uint4(0u, 0u, 0u, 0u);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) n_bits += __shfl_xor_sync(0xffffffffu, n_bits, o);
-  if (lane == 0) { s_cnt[wp] = n_pres; s_cnt[kRaWarps + wp] = n_bits; }
   __syncthreads();
-  int rank_run = 0, bits_run = 0;
-#pragma unroll
-  for (int i = 0; i < kRaWarps; ++i) {
-    rank_run += i < wp ? s_cnt[i] : 0;
-    bits_run += i < wp ? s_cnt[kRaWarps + i] : 0;
-  }
-  for (int i = 0; i < per; i += 32) {
-    const int kl = wp * per + i + lane;
-    const uint32_t m = mask[kl];
-    const unsigned bal = __ballot_sync(0xffffffffu, m != 0u);
-    const int pcnt = __popc(m);
-    int incl = pcnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += t;
-    }
-    if (m != 0u) {
-      const int first = bits_run + incl - pcnt;  // this row's first slot, relative to the range
-      info[kl] = (uint32_t)(rank_run + __popc(bal & lt)) | ((uint32_t)first << 13);
+  const uint32_t base_key = (uint32_t)(b << r_log2);
+  for_each_entry(ids, pc.entries, R, base_key, n_rows, s_beg, s_off, status,
+                 [&](int w, int, uint32_t, uint32_t kl) {
+                   atomicOr(&mask[kl], 1u << w);
+                   atomicOr(&pres[kl >> 5], 1u << (kl & 31));
+                 });
+  __syncthreads();
+
+  // thread q owns presence word q: present ids and contributions in it, prefix sums over the words
+  const uint32_t pw = tid < nW ? pres[tid] : 0u;
+  int n_ids = __popc(pw), n_con = 0;
+  for (uint32_t rest = pw; rest; rest &= rest - 1u) n_con += __popc(mask[tid * 32 + __ffs((int)rest) - 1]);
+  int tot_ids, tot_con;
+  block_scan2(n_ids, n_con, tot_ids, tot_con, s_tmp);  // now exclusive prefixes
+  if (tid < nW) {
+    wrank[tid] = n_ids;
+    int t = n_ids, first = n_con;
+    for (uint32_t rest = pw; rest; rest &= rest - 1u) {
+      first_c[t++] = (uint32_t)first;
       atomicOr(&hb[(hb_shift + first) >> 5], 1u << ((hb_shift + first) & 31));
+      first += __popc(mask[tid * 32 + __ffs((int)rest) - 1]);
     }
-    rank_run += __popc(bal);
-    bits_run += __shfl_sync(0xffffffffu, incl, 31);
   }
   __syncthreads();
 
@@ -296,37 +306,22 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
     if (g * 32 >= pc.before && g * 32 + 32 <= pc.before + pc.entries) head_bits[g] = word;
     else atomicOr(&head_bits[g], word);
   }
-  const uint32_t base_key = (uint32_t)(b << r_log2);
   const int64_t tile_mask = ((int64_t)1 << tile_shift) - 1;
-  for (int e0 = tid; e0 < pc.entries; e0 += kRaBatch * kRaThreads) {
-    int w[kRaBatch], j[kRaBatch];
-    uint32_t id[kRaBatch];
-#pragma unroll
-    for (int t = 0; t < kRaBatch; ++t) {
-      const int e = e0 + t * kRaThreads;
-      entry_of(e < pc.entries ? e : e0, s_beg, s_off, w[t], j[t]);
-      id[t] = (uint32_t)__ldg(ids + j[t]);
-    }
-#pragma unroll
-    for (int t = 0; t < kRaBatch; ++t) {
-      if (e0 + t * kRaThreads >= pc.entries) break;
-      const uint32_t kl = id[t] - base_key;
-      if (kl >= (uint32_t)R || (int64_t)id[t] >= n_rows) continue;  // flagged while building the table
-      const uint32_t m = mask[kl], inf = info[kl];
-      const int slot = __popc(m & ((1u << w[t]) - 1u));
-      const int64_t dest = pc.before + (int64_t)(inf >> 13) + slot;
-      const int64_t u = u0 + (int64_t)(inf & 0x1fffu);
-      src[dest] = (uint32_t)j[t];
-      if (slot == 0 && u < out_cap) agg_ids[u] = (int32_t)id[t];
-      if ((dest & tile_mask) == 0) tile_first[dest >> tile_shift] = (int32_t)u;
-    }
-  }
+  for_each_entry(ids, pc.entries, R, base_key, n_rows, s_beg, s_off, nullptr,
+                 [&](int w, int j, uint32_t id, uint32_t kl) {
+                   const int t = wrank[kl >> 5] + __popc(pres[kl >> 5] & ((1u << (kl & 31)) - 1u));
+                   const int slot = __popc(mask[kl] & ((1u << w) - 1u));
+                   const int64_t dest = pc.before + (int64_t)first_c[t] + slot;
+                   const int64_t u = u0 + t;
+                   src[dest] = (uint32_t)j;
+                   if (slot == 0 && u < out_cap) agg_ids[u] = (int32_t)id;
+                   if ((dest & tile_mask) == 0) tile_first[dest >> tile_shift] = (int32_t)u;
+                 });
 }
 
-size_t count_smem(int r_log2) { return 4 * ((size_t)1 << r_log2) + 8 + 4 * (32 + 33 + 8) + 12; }
 size_t emit_smem(int r_log2, int K) {  // tables, small arrays, head bits of up to R*K slots
   const size_t R = (size_t)1 << r_log2;
-  return 8 * R + 8 + 4 * (32 + 33 + 16) + 4 * (R * (size_t)K / 32 + 2) + 12;
+  return 8 * R + 8 + 4 * (256 + 256 + 32 + 33 + 16) + 4 * (R * (size_t)K / 32 + 2) + 12;
 }
 
 }  // namespace
@@ -370,7 +365,7 @@ void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t i
   ANTDT_LAUNCH("agg_range_split", range_split_kernel, (unsigned)((n_search + kRaThreads - 1) / kRaThreads),
                kRaThreads, 0, s, uniq_ids, wuo_in, K, in_cap, r_log2, P, dropped_bits, wuo_out, n_entries,
                bnd, status);
-  ANTDT_LAUNCH("agg_range_count", range_count_kernel, (unsigned)P, kRaThreads, count_smem(r_log2), s,
+  ANTDT_LAUNCH("agg_range_count", range_count_kernel, (unsigned)P, kRaThreads, 0, s,
                uniq_ids, bnd, wuo_out, K, P, r_log2, n_rows, dropped_bits, distinct, status);
   ANTDT_LAUNCH("agg_range_scan", range_scan_kernel, 1, 1024, 0, s, distinct, P, base, n_agg, out_cap,
                status);

@@ -14,15 +14,13 @@
 namespace antdt {
 
 constexpr int kRangeMaxWorkers = 32;        // one bit per worker in a 32-bit word
-constexpr int kRangeMinLog2 = 10;           // 1024 row ids per range at least
-constexpr int kRangeMaxLog2 = 13;           // 8192 at most (64 KB of shared memory)
+constexpr int kRangeLog2 = 12;              // 4096 row ids per range (measured best of 1024..8192)
+constexpr int kRangeMaxLog2 = 13;           // 8192 for tables beyond 2^30 rows (bounds the scratch)
 constexpr int64_t kRangeMaxRanges = (int64_t)1 << (31 - kRangeMaxLog2);  // n_rows < 2^31
 
-// log2 of the range width: about 32768 ranges over the table, within the limits above
+// log2 of the range width
 inline int range_log2(int64_t n_rows) {
-  int lg = kRangeMinLog2;
-  while (lg < kRangeMaxLog2 && ((int64_t)1 << (lg + 15)) < n_rows) ++lg;
-  return lg;
+  return n_rows > ((int64_t)kRangeMaxRanges << kRangeLog2) ? kRangeMaxLog2 : kRangeLog2;
 }
 
 struct RangeLayout {
