@@ -145,7 +145,7 @@ def plan_all(w, n_steps):
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
 # full-size default workload summarised in profiles/; a kernel that has changed since is set to None.
 NCU_TRAFFIC = {4: {"seg_reduce_tiles": 12.95e9, "agg_reduce": 6.80e9, "sparse_adagrad": 9.42e9,
-                   "embbag_fwd": 4.04e9, "radix_scatter": (2.96e9 + 2.39e9 + 2.11e9) / 3}}
+                   "embbag_fwd": 4.04e9, "radix_scatter": (2.90e9 + 2.34e9 + 2.08e9) / 3}}
 
 
 def scaled_workload(w, scale):
@@ -167,6 +167,9 @@ def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
         "runs_emit": 4 * nnz + nnz // 8 + 12 * sum_u,
         "agg_radix_hist": 4 * sum_u, "agg_radix_scatter": 16 * sum_u, "agg_runs_count": 4 * sum_u,
         "agg_runs_emit": 4 * sum_u + sum_u // 8 + 12 * u,
+        # range-partitioned merge (up to 32 workers): ids read by both passes; merge order, head
+        # bits and the distinct ids written once
+        "agg_range_count": 4 * sum_u, "agg_range_emit": 8 * sum_u + sum_u // 8 + 4 * u,
         "embbag_fwd": 4 * nnz + 8 * (n_bags + 1) + nnz * D * ew + n_bags * D * 4,
         "expand_bags": 8 * (n_bags + 1) + 4 * nnz,
         "seg_reduce_tiles": 4 * nnz + nnz // 8 + nnz * D * 4 + sum_u * D * 4,
@@ -180,9 +183,12 @@ def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
 def step_bytes(w, nnz, n_bags, sum_u, u, passes_bwd, passes_agg):
     b = algorithmic_bytes(w, nnz, n_bags, sum_u, u)
     upd = b["sparse_adam"] if w.opt == "adam" else b["sparse_adagrad"]
-    sort = (passes_bwd * (b["radix_hist"] + b["radix_scatter"]) + b["runs_count"] + b["runs_emit"] +
-            passes_agg * (b["agg_radix_hist"] + b["agg_radix_scatter"]) + b["agg_runs_count"] +
-            b["agg_runs_emit"])
+    sort = passes_bwd * (b["radix_hist"] + b["radix_scatter"]) + b["runs_count"] + b["runs_emit"]
+    if w.K <= 32:       # the aggregation's merge order comes from the range pass, not a sort
+        sort += b["agg_range_count"] + b["agg_range_emit"]
+    else:
+        sort += (passes_agg * (b["agg_radix_hist"] + b["agg_radix_scatter"]) + b["agg_runs_count"] +
+                 b["agg_runs_emit"])
     return (b["embbag_fwd"] + b["expand_bags"] + b["seg_reduce_tiles"] + b["agg_reduce"] + upd +
             (b["dense_wsum"] if w.dense_n else 0) + sort)
 
