@@ -183,6 +183,74 @@ def test_sparse_aggregate_matches_checker(V, D, K, n_per):
     G.close(agg, want)
 
 
+def _lists_case(rng, K, make):
+    lists = [np.unique(make(i)).astype(np.int64) for i in range(K)]
+    uid = np.concatenate(lists).astype(np.int32)
+    wuo = np.concatenate([[0], np.cumsum([len(l) for l in lists])]).astype(np.int64)
+    return uid, wuo
+
+
+def test_sparse_aggregate_clustered_and_dense_ranges():
+    """Row ids that are NOT spread by a hash: every worker holds the same dense block (every
+    4096-id range of it carries K entries per id), plus a thin tail; 32 workers fill every bit of
+    the worker-set words; dim 4 puts one lane on a row."""
+    rng = np.random.default_rng(61)
+    for K, D, dense_to, V in [(32, 4, 20_000, 3_000_000), (8, 32, 70_000, 200_000), (17, 16, 9000, 9001)]:
+        def make(i):
+            tail = rng.integers(dense_to, V, size=500) if V > dense_to else np.zeros(0, np.int64)
+            keep = rng.random(dense_to) < (1.0 if i % 3 == 0 else 0.8)
+            return np.concatenate([np.nonzero(keep)[0], tail])
+        uid, wuo = _lists_case(rng, K, make)
+        g = rng.normal(size=(len(uid), D)).astype(np.float32)
+        bsz = rng.integers(1, 4000, size=K)
+        ids, agg, na, _, code = G.gpu_aggregate(uid, wuo, g, bsz, V)
+        assert code == 0
+        want_ids, want = oracle.aggregate_sparse(uid, wuo, g, bsz)
+        assert na == len(want_ids) and np.array_equal(ids, want_ids)
+        G.close(agg, want)
+
+
+def test_sparse_aggregate_table_beyond_2_to_30_rows():
+    """n_rows above 2^30 switches the merge to 8192-id ranges (the row count is only a bound here:
+    no table is touched).  Ids sit at both ends of the id space and around a range boundary."""
+    rng = np.random.default_rng(62)
+    V = (1 << 31) - 1
+    K, D = 6, 16
+    edge = np.array([0, 1, 8191, 8192, 8193, V - 8193, V - 2, V - 1], np.int64)
+
+    def make(i):
+        return np.concatenate([edge[rng.random(len(edge)) < 0.7], rng.integers(0, V, size=20_000),
+                               rng.integers(1 << 30, (1 << 30) + 50_000, size=10_000)])
+    uid, wuo = _lists_case(rng, K, make)
+    g = rng.normal(size=(len(uid), D)).astype(np.float32)
+    bsz = rng.integers(1, 4000, size=K)
+    ids, agg, na, _, code = G.gpu_aggregate(uid, wuo, g, bsz, V)
+    assert code == 0
+    want_ids, want = oracle.aggregate_sparse(uid, wuo, g, bsz)
+    assert na == len(want_ids) and np.array_equal(ids, want_ids)
+    G.close(agg, want)
+
+
+def test_sparse_aggregate_flags_ids_outside_the_table():
+    """An id >= n_rows is not part of the union: flagged, skipped, and every access stays inside
+    the buffers (whatever else the flagged call returns is unspecified)."""
+    rng = np.random.default_rng(63)
+    V, K, D = 50_000, 4, 8
+    uid, wuo = _lists_case(rng, K, lambda i: rng.integers(0, V, size=3000))
+    g = rng.normal(size=(len(uid), D)).astype(np.float32)
+    bad = uid.copy()
+    bad[wuo[2] - 1] = V + 5            # last (largest) id of worker 1's list: still ascending
+    _, _, _, _, code = G.gpu_aggregate(bad, wuo, g, [1] * K, V)
+    assert code == B.ERR_ID_OUT_OF_RANGE
+    bad[wuo[2] - 1] = 60_000_000       # far past the last range of the table
+    _, _, _, _, code = G.gpu_aggregate(bad, wuo, g, [1] * K, V)
+    assert code == B.ERR_ID_OUT_OF_RANGE
+    ids, agg, na, _, code = G.gpu_aggregate(uid, wuo, g, [1] * K, V)   # the clean lists still work
+    want_ids, want = oracle.aggregate_sparse(uid, wuo, g, [1] * K)
+    assert code == 0 and np.array_equal(ids, want_ids)
+    G.close(agg, want)
+
+
 def test_aggregate_invariants_on_gpu():
     rng = np.random.default_rng(21)
     V, D, F, K, S = 300, 16, 3, 4, 512
