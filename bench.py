@@ -89,6 +89,14 @@ class ClockSampler:
         except OSError:
             self.p = None
 
+    def count(self):
+        """Samples written so far."""
+        try:
+            with open(self.f.name) as g:
+                return sum(1 for ln in g if ln.strip())
+        except OSError:
+            return 0
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
@@ -358,17 +366,27 @@ def run_ours(args):
     torch.cuda.synchronize()
     stream = torch.cuda.Stream() if use_graph else torch.cuda.current_stream()
     torch.cuda.set_stream(stream)
+    # the sampler runs from before the warm-up to after the timed region: a timed region of a few
+    # milliseconds (small configurations) would otherwise fall between two samples
+    clocks = ClockSampler(local_rank)
+    clocks.start()
     for s in range(W):
         one_step(s)
+    # nvidia-smi takes a moment to deliver its first sample: keep stepping (untimed) until it has,
+    # so that the clocks are seen under this load even when the timed region lasts milliseconds
+    extra, t_wait = 0, time.time()
+    while clocks.p is not None and clocks.count() < 2 and time.time() - t_wait < 3.0:
+        one_step(W + extra)
+        extra += 1
+        if extra % 8 == 0:
+            torch.cuda.synchronize()
     torch.cuda.synchronize()
     assert B.antdt_read_status(buf.status) == 0, "device status after warm-up"
     u_seen = int(buf.n_agg.item())
     sum_u_seen = int(buf.worker_uniq_offsets[w.K].item())
 
-    clocks = ClockSampler(local_rank)
     barrier()
     torch.cuda.synchronize()
-    clocks.start()
     if not use_graph:
         B.antdt_profile_enable(True)    # an event pair around every launch of the timed steps
     launches0 = B.antdt_launch_count()
@@ -439,7 +457,13 @@ def run_ours(args):
         roof["frac"] = round(roof["achieved"] / peak_gbs, 4)
     if top in ("seg_reduce_tiles", "embbag_fwd"):
         roof["note"] = ("gather counted at full multiplicity; repeats of a row are served by L2, so the "
-                        "algorithmic rate can exceed the DRAM peak: see traffic")
+                        "algorithmic rate can exceed the DRAM peak: see traffic and the compulsory figures")
+        # every distinct input row once + ids + outputs: what a perfect cache would leave for DRAM
+        D, ew = w.D, (2 if w.table_dtype == "bf16" else 4)
+        comp = (4 * nnz_avg + nnz_avg / 8 + bags_avg * D * 4 + sum_u_seen * D * 4 if top == "seg_reduce_tiles"
+                else 4 * nnz_avg + 8 * (bags_avg + 1) + u_seen * D * ew + bags_avg * D * 4)
+        roof["compulsory_bytes_per_launch"] = int(comp)
+        roof["frac_compulsory"] = round(comp / (top_ms / top_n * 1e-3) / 1e9 / peak_gbs, 4)
     if args.scale == 1.0 and world == 1:
         roof["traffic"] = NCU_TRAFFIC.get(cfg, {}).get(top)
         if roof["traffic"]:
@@ -460,7 +484,8 @@ def run_ours(args):
                    "launch": ("one CUDA graph per step (antdt_bsp_step_graph)" if use_graph
                               else "plain launches (antdt_bsp_step_device)"),
                    "parallelism": "replicas" if world > 1 else "single"},
-        "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"]},
+        "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"],
+                   "samples": clk["samples"], "extra_warmup_steps": extra},
         "e2e": None if args.no_e2e else {
             "value": e2e_samples / (e2e_ms * 1e-3), "unit": UNIT,
             "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
