@@ -212,9 +212,17 @@ int32_t antdt_embbag_fwd(const void* table, int32_t dtype, int64_t n_rows, int32
  *                        (worker, row id, then original position: all three unique)
  *   uniq_grads           device out [out_cap, dim] fp32
  *   out_cap              capacity in rows; nnz always suffices; CAPACITY -> dev_status
- *   ws, ws_bytes         device scratch >= antdt_embbag_bwd_dedup_workspace_bytes(...) */
+ *   ws, ws_bytes         device scratch.  antdt_embbag_bwd_dedup_workspace_bytes(...) is the size
+ *                        to allocate; antdt_embbag_bwd_dedup_min_workspace_bytes(...) is the least
+ *                        the call accepts (WORKSPACE_TOO_SMALL below it).  The two differ for up to
+ *                        2^20 occurrences only: with the larger one the reduction walks 16-entry
+ *                        tiles, which keeps a small input spread over the whole GPU; with less it
+ *                        walks the 64-entry tiles of large inputs.  Results are the same up to the
+ *                        order of the floating-point sums (both orders are fixed). */
 size_t antdt_embbag_bwd_dedup_workspace_bytes(int64_t nnz, int64_t n_bags, int32_t dim,
                                               int32_t n_workers);
+size_t antdt_embbag_bwd_dedup_min_workspace_bytes(int64_t nnz, int64_t n_bags, int32_t dim,
+                                                  int32_t n_workers);
 int32_t antdt_embbag_bwd_dedup(const int32_t* row_ids, int64_t nnz, const int64_t* bag_offsets,
                                int64_t n_bags, int32_t bags_per_sample, const float* d_pooled,
                                int32_t dim, int64_t n_rows, int32_t n_workers,
@@ -233,7 +241,7 @@ int32_t antdt_embbag_bwd_dedup(const int32_t* row_ids, int64_t nnz, const int64_
  * the library holds it from load to exit, whether or not this call is ever used.
  *   - Arguments and results are those of antdt_embbag_bwd_dedup without ws / ws_bytes; inputs and
  *     outputs are still the caller's buffers.
- *   - Limit: antdt_embbag_bwd_dedup_workspace_bytes(nnz, n_bags, dim, n_workers) must not exceed
+ *   - Limit: antdt_embbag_bwd_dedup_min_workspace_bytes(nnz, n_bags, dim, n_workers) must not exceed
  *     ANTDT_STATIC_SCRATCH_BYTES (24 MiB: roughly 1.1 million occurrences at dim 64, 1.7 million at
  *     dim 16, with up to 64 workers).  Beyond it the call returns ANTDT_ERR_CAPACITY and launches
  *     nothing.

@@ -29,7 +29,8 @@ EXPORTS = [
     "antdt_dds_requeue_worker", "antdt_dds_num_shards", "antdt_dds_counts", "antdt_dds_shard_info",
     "antdt_dds_save", "antdt_dds_load", "antdt_ctl_create", "antdt_ctl_destroy",
     "antdt_ctl_report", "antdt_ctl_decide", "antdt_dd_solve", "antdt_embbag_fwd",
-    "antdt_embbag_bwd_dedup_workspace_bytes", "antdt_embbag_bwd_dedup",
+    "antdt_embbag_bwd_dedup_workspace_bytes", "antdt_embbag_bwd_dedup_min_workspace_bytes",
+    "antdt_embbag_bwd_dedup",
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
     "antdt_weighted_aggregate_backup",
@@ -116,6 +117,8 @@ def lib() -> C.CDLL:
         L.antdt_embbag_fwd.argtypes = [P, I32, I64, I32, P, I64, P, I64, P, P, P]
         L.antdt_embbag_bwd_dedup_workspace_bytes.argtypes = [I64, I64, I32, I32]
         L.antdt_embbag_bwd_dedup_workspace_bytes.restype = SZ
+        L.antdt_embbag_bwd_dedup_min_workspace_bytes.argtypes = [I64, I64, I32, I32]
+        L.antdt_embbag_bwd_dedup_min_workspace_bytes.restype = SZ
         L.antdt_embbag_bwd_dedup.argtypes = [P, I64, P, I64, I32, P, I32, I64, I32, P, P, P, P, P, P,
                                              I64, P, SZ, P, P]
         L.antdt_embbag_bwd_dedup_static.argtypes = [P, I64, P, I64, I32, P, I32, I64, I32, P, P, P, P,
@@ -316,6 +319,10 @@ def antdt_embbag_fwd(table, row_ids, bag_offsets, pooled, dev_status=None, strea
 
 def antdt_embbag_bwd_dedup_workspace_bytes(nnz: int, n_bags: int, dim: int, n_workers: int) -> int:
     return lib().antdt_embbag_bwd_dedup_workspace_bytes(nnz, n_bags, dim, n_workers)
+
+
+def antdt_embbag_bwd_dedup_min_workspace_bytes(nnz: int, n_bags: int, dim: int, n_workers: int) -> int:
+    return lib().antdt_embbag_bwd_dedup_min_workspace_bytes(nnz, n_bags, dim, n_workers)
 
 
 def antdt_embbag_bwd_dedup(row_ids, bag_offsets, bags_per_sample: int, d_pooled, n_rows: int,

@@ -41,7 +41,8 @@ AggLayout agg_layout(int64_t in_cap, int K, int dim) {
   L.src = o;       o = align_up(o + 4 * n);
   L.vals_t = o;    o = align_up(o + 4 * n);
   L.run_start = o; o = align_up(o + 8 * (n + 1));
-  const size_t n_tiles = (n + kRedTile - 1) / kRedTile;
+  const size_t tile = (size_t)red_tile_for((int64_t)n);
+  const size_t n_tiles = (n + tile - 1) / tile;
   L.head_bits = o;  o = align_up(o + 4 * head_bits_words((int64_t)n));
   L.tile_first = o; o = align_up(o + 4 * (n_tiles + 1));
   L.head_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
@@ -216,7 +217,7 @@ void sort_merge_order(const antdt_sparse_part* sp, const uint8_t* dropped, bool 
                 (uint32_t*)(w8 + L.vals_t), key_bits, 0, sort_ws, L.sort, dev_status, s, true);
     segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
                  agg_cap, (uint32_t*)(w8 + L.head_bits),
-                 (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws, L.sort, dev_status, s, true);
+                 (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap > 0 ? in_cap : 1), sort_ws, L.sort, dev_status, s, true);
 }
 
 int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
@@ -270,7 +271,7 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
       range_merge_order(sp->uniq_ids, sp->worker_uniq_offsets, in_cap, sp->n_rows, K, dropped_bits,
                         sp->agg_ids, sp->n_agg, agg_cap, (int64_t*)(w8 + L.wuo), bounds,
                         (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.head_bits),
-                        (int32_t*)(w8 + L.tile_first), kRedTile, w8 + L.range_ws, L.range, dev_status, s);
+                        (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap), w8 + L.range_ws, L.range, dev_status, s);
     } else {
       sort_merge_order(sp, dropped, any_dropped, K, in_cap, agg_cap, w8, L, dev_status, s);
     }
@@ -279,6 +280,7 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
       t.payload = (const uint32_t*)(w8 + L.src);
       t.head_bits = (const uint32_t*)(w8 + L.head_bits);
       t.tile_first = (const int32_t*)(w8 + L.tile_first);
+      t.tile = red_tile_for(in_cap);
       t.rows = sp->uniq_grads;
       t.dim = sp->dim;
       t.n_host = in_cap;

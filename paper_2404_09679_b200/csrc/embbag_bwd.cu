@@ -8,7 +8,7 @@
 //   reduce    tile-parallel segmented sum of gathered d_pooled rows
 //   fixup     rows whose occurrences straddle tiles: ordered sum of the tiles' partials
 //
-// The reduction is balanced by occurrences, not by rows: a tile is kRedTile consecutive
+// The reduction is balanced by occurrences, not by rows: a tile is 64 (small inputs: 16) consecutive
 // sorted occurrences whatever rows they belong to, so a row that holds 20% of a field's
 // occurrences costs its tiles no more than anyone else's.  Every sum has a fixed order (inside a
 // tile by sorted position, across tiles by tile index), no floating-point atomics anywhere.
@@ -26,11 +26,12 @@ struct BwdLayout {
       head_part, tail_part, bytes;
 };
 
-BwdLayout bwd_layout(int64_t nnz, int dim, int K) {
+BwdLayout bwd_layout(int64_t nnz, int dim, int K, int tile_len) {
   BwdLayout L;
   L.sort = sort_layout(K);
   const size_t n = (size_t)(nnz > 0 ? nnz : 1);
-  const size_t n_tiles = (n + kRedTile - 1) / kRedTile;
+  const size_t tile = (size_t)tile_len;
+  const size_t n_tiles = (n + tile - 1) / tile;
   size_t o = 0;
   L.sort_ws = o;    o = align_up(o + L.sort.bytes);
   L.wso = o;        o = align_up(o + 8 * ((size_t)K + 1));
@@ -102,7 +103,14 @@ extern "C" size_t antdt_embbag_bwd_dedup_workspace_bytes(int64_t nnz, int64_t n_
                                                          int32_t n_workers) {
   (void)n_bags;
   if (nnz < 0 || dim < 1 || n_workers < 1 || n_workers > antdt::kMaxSegments) return 0;
-  return antdt::bwd_layout(nnz, dim, n_workers).bytes;
+  return antdt::bwd_layout(nnz, dim, n_workers, antdt::red_tile_for(nnz)).bytes;
+}
+
+extern "C" size_t antdt_embbag_bwd_dedup_min_workspace_bytes(int64_t nnz, int64_t n_bags, int32_t dim,
+                                                             int32_t n_workers) {
+  (void)n_bags;
+  if (nnz < 0 || dim < 1 || n_workers < 1 || n_workers > antdt::kMaxSegments) return 0;
+  return antdt::bwd_layout(nnz, dim, n_workers, antdt::kRedTile).bytes;
 }
 
 namespace antdt {
@@ -129,7 +137,14 @@ int32_t bwd_dedup_impl(
   for (int w = 0; w < K; ++w)
     if (worker_sample_offsets[w + 1] < worker_sample_offsets[w]) return ANTDT_ERR_INVALID_ARG;
   if (worker_sample_offsets[K] * (int64_t)bags_per_sample != n_bags) return ANTDT_ERR_INVALID_ARG;
-  const BwdLayout L = bwd_layout(nnz, dim, K);
+  // short reduction tiles for a small input when the workspace has room for their partial sums,
+  // the long tiles (the minimum workspace) otherwise
+  int tile_len = red_tile_for(nnz);
+  BwdLayout L = bwd_layout(nnz, dim, K, tile_len);
+  if (ws_bytes < L.bytes && tile_len != kRedTile) {
+    tile_len = kRedTile;
+    L = bwd_layout(nnz, dim, K, tile_len);
+  }
   if (ws_bytes < L.bytes) return ANTDT_ERR_WORKSPACE_TOO_SMALL;
 
   cudaStream_t s = (cudaStream_t)stream;
@@ -160,7 +175,7 @@ int32_t bwd_dedup_impl(
   segsort_run(reinterpret_cast<const uint32_t*>(row_ids), expand_to, keys_a, occ_out, keys_b,
               vals_t, key_bits, n_rows, sort_ws, L.sort, dev_status, s);
   segsort_runs(keys_a, nnz, uniq_ids, seg_offsets, worker_uniq_offsets, nullptr, out_cap,
-               (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), kRedTile, sort_ws,
+               (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), tile_len, sort_ws,
                L.sort, dev_status, s);
   if (d_pooled_ready && cudaStreamWaitEvent(s, d_pooled_ready, 0) != cudaSuccess)
     return ANTDT_ERR_CUDA;
@@ -169,6 +184,7 @@ int32_t bwd_dedup_impl(
     t.payload = occ_out;
     t.head_bits = (const uint32_t*)(w8 + L.head_bits);
     t.tile_first = (const int32_t*)(w8 + L.tile_first);
+    t.tile = tile_len;
     t.rows = d_pooled;
     t.dim = dim;
     t.n_host = nnz;

@@ -27,7 +27,7 @@ extern "C" int32_t antdt_embbag_bwd_dedup_static(
     int64_t* seg_offsets, int32_t* sorted_occ, float* uniq_grads, int64_t out_cap,
     int32_t* dev_status, void* stream) {
   // size check first: nothing is launched for a problem the fixed array cannot hold
-  const size_t need = antdt_embbag_bwd_dedup_workspace_bytes(nnz, n_bags, dim, n_workers);
+  const size_t need = antdt_embbag_bwd_dedup_min_workspace_bytes(nnz, n_bags, dim, n_workers);
   if (need == 0) return ANTDT_ERR_INVALID_ARG;
   if (need > (size_t)ANTDT_STATIC_SCRATCH_BYTES) return ANTDT_ERR_CAPACITY;
 

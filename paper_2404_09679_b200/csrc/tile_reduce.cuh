@@ -2,8 +2,8 @@
 // d_pooled rows per (worker, row) run, scaled by 1/b_w) and the server aggregation (weighted sum
 // of the workers' gradient rows per row).
 //
-// The sorted array of payloads (row indices into `rows`) is cut into tiles of kRedTile = 64
-// consecutive entries whatever runs they belong to, so the work is balanced by entries, not by
+// The sorted array of payloads (row indices into `rows`) is cut into tiles of 64 (16 for a small
+// input) consecutive entries whatever runs they belong to, so the work is balanced by entries, not by
 // runs: a run holding 20% of a field costs its tiles no more than anyone else's.  A group of G
 // lanes (one 16-byte vector of the row per lane and VPL step) walks one tile; a run that starts
 // and ends inside the tile is written out, the pieces of runs that cross the tile's edges go to
@@ -21,14 +21,20 @@
 
 namespace antdt {
 
-constexpr int kRedTile = 64;  // sorted entries per reduction tile (a power of two, multiple of 32)
+constexpr int kRedTile = 64;       // sorted entries per reduction tile of a large input
+constexpr int kRedTileSmall = 16;  // ... of a small one: a tile is walked serially, so a small input
+                                   // needs short tiles to fill the machine and to end soon
+constexpr int64_t kRedSmallN = (int64_t)1 << 20;
+// Tile length for an input of at most n entries (n: the host-side bound the launch is sized by).
+inline int red_tile_for(int64_t n) { return n <= kRedSmallN ? kRedTileSmall : kRedTile; }
 constexpr int kRedThreads = 256;
 constexpr int kRedUnroll = 4;
 
 struct TileArgs {
   const uint32_t* payload;    // [n] sorted payloads: row index into `rows`
   const uint32_t* head_bits;  // bit i set iff entry i starts a run
-  const int32_t* tile_first;  // run index of entry t*kRedTile
+  const int32_t* tile_first;  // run index of entry t*tile
+  int tile;                   // red_tile_for(n_host)
   const float* rows;          // gathered matrix [payload_limit, dim]
   int dim;
   int64_t n_host;             // entries (upper bound when n_dev is given)
@@ -46,7 +52,7 @@ struct TileArgs {
 
 // The hot pointers are separate __restrict__ parameters (not read through the struct) so that
 // the compiler may move row loads across the run-end stores.
-template <int G, int VPL, bool AGG>
+template <int G, int VPL, bool AGG, int TILE>
 __global__ void __launch_bounds__(kRedThreads, (VPL == 1 ? 6 : 1))
 tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
                    const uint32_t* __restrict__ head_bits, const int32_t* __restrict__ tile_first,
@@ -62,32 +68,41 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
   const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
   const int lg = threadIdx.x & (G - 1);
   const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
-  const int64_t o_begin = tile * kRedTile;
+  const int64_t o_begin = tile * TILE;
   if (o_begin >= n) return;
-  const int nv = (int)min((int64_t)kRedTile, n - o_begin);  // entries in this tile
+  const int nv = (int)min((int64_t)TILE, n - o_begin);  // entries in this tile
   const unsigned gmask = group_mask<G>();
   const int dim = a.dim;
   const int nvec = dim / 4;
   constexpr int U = (G < kRedUnroll) ? G : kRedUnroll;
 
-  // run heads of positions o_begin .. o_begin+64; entry r closes its run iff r+1 is a head
+  // run heads of positions o_begin .. o_begin+TILE; entry r closes its run iff r+1 is a head
   const uint32_t* hw = head_bits + (o_begin >> 5);
-  const uint32_t h0 = __ldg(hw), h1 = __ldg(hw + 1), h2 = __ldg(hw + 2);
-  const uint64_t heads = (uint64_t)h0 | ((uint64_t)h1 << 32);
-  uint64_t ends = (heads >> 1) | ((uint64_t)(h2 & 1u) << 63);
-  const bool last_tile = o_begin + kRedTile >= n;
+  const bool last_tile = o_begin + TILE >= n;
+  uint64_t ends;
+  bool open_tail, started;
+  if (TILE == 64) {
+    const uint32_t h0 = __ldg(hw), h1 = __ldg(hw + 1), h2 = __ldg(hw + 2);
+    const uint64_t heads = (uint64_t)h0 | ((uint64_t)h1 << 32);
+    ends = (heads >> 1) | ((uint64_t)(h2 & 1u) << 63);
+    open_tail = !last_tile && !(h2 & 1u);  // the last run goes on in the next tile
+    started = (h0 & 1u) != 0;
+  } else {  // TILE < 32 and a power of two: the tile's bits and the next one lie in two words
+    const uint64_t heads = ((uint64_t)__ldg(hw) | ((uint64_t)__ldg(hw + 1) << 32)) >> (o_begin & 31);
+    ends = (heads >> 1) & ((1ull << TILE) - 1ull);
+    open_tail = !last_tile && !((heads >> TILE) & 1ull);
+    started = (heads & 1ull) != 0;
+  }
   if (last_tile) ends = (ends & ((1ull << (nv - 1)) - 1ull)) | (1ull << (nv - 1));  // array end closes
-  const bool open_tail = !last_tile && !(h2 & 1u);  // the last run goes on in the next tile
 
   int64_t u = tile_first[tile];
-  bool started = (h0 & 1u) != 0;
-  int w = 0, next_w_rel = kRedTile + 1;
+  int w = 0, next_w_rel = TILE + 1;
   float inv = 1.f;
   if (!AGG) {
     w = interval_of(s_bounds, K + 1, o_begin);
     if (w > K - 1) w = K - 1;
     // tile-relative position at which the next worker starts (beyond the tile: never reached)
-    next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
+    next_w_rel = (int)min((int64_t)(TILE + 1), s_bounds[w + 1] - o_begin);
     inv = a.scales[w];
   }
 
@@ -143,8 +158,8 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
               if (rel >= next_w_rel) {  // crossed into a later worker's range
                 const int64_t o = o_begin + rel;
                 while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
-                next_w_rel = (int)min((int64_t)(kRedTile + 1), s_bounds[w + 1] - o_begin);
-                if (w == K - 1) next_w_rel = kRedTile + 1;
+                next_w_rel = (int)min((int64_t)(TILE + 1), s_bounds[w + 1] - o_begin);
+                if (w == K - 1) next_w_rel = TILE + 1;
                 inv = a.scales[w];
               }
               sc = inv;
@@ -182,17 +197,30 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
   }
 }
 
+// Head bits of the TILE entries from pos (a multiple of TILE), and the single bit at pos.
+template <int TILE>
+__device__ __forceinline__ uint64_t tile_heads(const uint32_t* __restrict__ hb, int64_t pos) {
+  if (TILE == 64) {
+    const uint32_t* w = hb + (pos >> 5);
+    return (uint64_t)__ldg(w) | ((uint64_t)__ldg(w + 1) << 32);
+  }
+  return (uint64_t)(__ldg(hb + (pos >> 5)) >> (pos & 31)) & ((1ull << (TILE & 63)) - 1ull);  // inside one word
+}
+__device__ __forceinline__ bool head_at(const uint32_t* __restrict__ hb, int64_t pos) {
+  return ((__ldg(hb + (pos >> 5)) >> (pos & 31)) & 1u) != 0u;
+}
+
 // Fix-up: the tile in which a straddling run STARTS owns it.  total = its tail piece, then
 // the head pieces of the following tiles in order until the run ends.
-template <int G, int VPL, bool AGG>
+template <int G, int VPL, bool AGG, int TILE>
 __global__ void __launch_bounds__(kRedThreads)
 tile_fixup_kernel(const TileArgs a) {
   const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
   const int lg = threadIdx.x & (G - 1);
   const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
-  const int64_t o_begin = tile * kRedTile;
+  const int64_t o_begin = tile * TILE;
   if (o_begin >= n) return;
-  const int64_t o_end = o_begin + kRedTile;
+  const int64_t o_end = o_begin + TILE;
   if (o_end >= n) return;  // the last tile's runs all end inside it
   const int dim = a.dim;
   const int nvec = dim / 4;
@@ -200,10 +228,9 @@ tile_fixup_kernel(const TileArgs a) {
   // depends on the tile index is requested up front: the head bits of this tile and the next
   // (a straddling run nearly always ends there), the run index, this tile's tail piece and the
   // next tile's head piece.  (The mask and the partial arrays reach one tile past the end.)
-  constexpr int kW = kRedTile / 32;
-  uint32_t hb[2 * kW + 1];
-#pragma unroll
-  for (int i = 0; i <= 2 * kW; ++i) hb[i] = __ldg(a.head_bits + (o_begin >> 5) + i);
+  const uint64_t cur = tile_heads<TILE>(a.head_bits, o_begin);
+  const uint64_t nxt_heads = tile_heads<TILE>(a.head_bits, o_end);
+  const bool after = head_at(a.head_bits, o_end + TILE);
   const int32_t first_run = __ldg(a.tile_first + tile);
   float4 tot[VPL], nxt[VPL];
 #pragma unroll
@@ -221,12 +248,10 @@ tile_fixup_kernel(const TileArgs a) {
     if (w > a.K - 1) w = a.K - 1;
     scale = a.scales[w];
   }
-  if (hb[kW] & 1u) return;  // next tile starts a new run: nothing straddles
-  int heads = 0;
-#pragma unroll
-  for (int i = 0; i < kW; ++i) heads += __popc(hb[i]);
+  if (nxt_heads & 1ull) return;  // next tile starts a new run: nothing straddles
+  const int heads = __popcll(cur);
   if (heads == 0) return;  // the straddling run started earlier: its start tile owns it
-  const int64_t u = (int64_t)first_run + heads - ((hb[0] & 1u) ? 1 : 0);
+  const int64_t u = (int64_t)first_run + heads - ((cur & 1ull) ? 1 : 0);
   if (u >= a.out_cap) return;
 
 #pragma unroll
@@ -234,12 +259,9 @@ tile_fixup_kernel(const TileArgs a) {
     tot[k].x += nxt[k].x; tot[k].y += nxt[k].y; tot[k].z += nxt[k].z; tot[k].w += nxt[k].w;
   }
   // does the run go on past tile+1?  (no head inside it nor at the start of the tile after it)
-  bool open = o_end + kRedTile < n;
-#pragma unroll
-  for (int i = kW; i < 2 * kW; ++i) open = open && hb[i] == 0u;
-  open = open && (hb[2 * kW] & 1u) == 0u;
+  bool open = o_end + TILE < n && nxt_heads == 0ull && !after;
   for (int64_t t2 = tile + 2; open; ++t2) {
-    const int64_t b2 = t2 * kRedTile;
+    const int64_t b2 = t2 * TILE;
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
       const int vi = lg + k * G;
@@ -247,12 +269,9 @@ tile_fixup_kernel(const TileArgs a) {
       const float4 p = reinterpret_cast<const float4*>(a.head_part + (size_t)t2 * dim)[vi];
       tot[k].x += p.x; tot[k].y += p.y; tot[k].z += p.z; tot[k].w += p.w;
     }
-    if (b2 + kRedTile >= n) break;  // ran to the end of the array
-    bool ends = false;              // a head inside t2, or at the start of the tile after it
-#pragma unroll
-    for (int i = 0; i < kW; ++i) ends |= __ldg(a.head_bits + (b2 >> 5) + i) != 0u;
-    ends |= (__ldg(a.head_bits + (b2 >> 5) + kW) & 1u) != 0u;
-    if (ends) break;
+    if (b2 + TILE >= n) break;  // ran to the end of the array
+    // a head inside t2, or at the start of the tile after it, ends the run
+    if (tile_heads<TILE>(a.head_bits, b2) != 0ull || head_at(a.head_bits, b2 + TILE)) break;
   }
   float* dst = a.out + (size_t)u * dim;
 #pragma unroll
@@ -265,17 +284,24 @@ tile_fixup_kernel(const TileArgs a) {
   }
 }
 
-template <int G, int VPL, bool AGG>
-void launch_tile_reduce_gv(const TileArgs& a, const char* name_tiles, const char* name_fixup,
-                           cudaStream_t s) {
-  const int64_t n_tiles = (a.n_host + kRedTile - 1) / kRedTile;
+template <int G, int VPL, bool AGG, int TILE>
+void launch_tile_reduce_t(const TileArgs& a, const char* name_tiles, const char* name_fixup,
+                          cudaStream_t s) {
+  const int64_t n_tiles = (a.n_host + TILE - 1) / TILE;
   const int64_t tpb = kRedThreads / G;
   const unsigned grid = (unsigned)((n_tiles + tpb - 1) / tpb);
   if (grid == 0) return;
   const size_t smem = 8 * ((size_t)a.K + 1) + (AGG ? 4 * (size_t)a.K : 0);
-  ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, AGG>), grid, kRedThreads, smem, s, a, a.payload,
-               a.head_bits, a.tile_first, a.rows, a.out, a.head_part, a.tail_part);
-  ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, AGG>), grid, kRedThreads, 0, s, a);
+  ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, smem, s, a,
+               a.payload, a.head_bits, a.tile_first, a.rows, a.out, a.head_part, a.tail_part);
+  ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, 0, s, a);
+}
+
+template <int G, int VPL, bool AGG>
+void launch_tile_reduce_gv(const TileArgs& a, const char* name_tiles, const char* name_fixup,
+                           cudaStream_t s) {
+  if (a.tile == kRedTileSmall) launch_tile_reduce_t<G, VPL, AGG, kRedTileSmall>(a, name_tiles, name_fixup, s);
+  else launch_tile_reduce_t<G, VPL, AGG, kRedTile>(a, name_tiles, name_fixup, s);
 }
 
 template <bool AGG>

@@ -68,7 +68,7 @@ def gpu_fwd(table_np, ids, off, status=None):
     return pooled[:n_bags].cpu().numpy(), code
 
 
-def gpu_bwd(ids, off, F, dY, n_rows, wso, out_cap=None):
+def gpu_bwd(ids, off, F, dY, n_rows, wso, out_cap=None, min_workspace=False):
     nnz, n_bags, D, K = ids.shape[0], off.shape[0] - 1, dY.shape[1], len(wso) - 1
     cap = max(1, nnz if out_cap is None else out_cap)
     uid = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
@@ -76,8 +76,9 @@ def gpu_bwd(ids, off, F, dY, n_rows, wso, out_cap=None):
     so = torch.full((cap + 1,), -1, dtype=torch.int64, device="cuda")
     occ = torch.full((max(nnz, 1),), -1, dtype=torch.int32, device="cuda")
     ug = torch.full((cap, D), float("nan"), device="cuda")
-    ws = torch.empty(B.antdt_embbag_bwd_dedup_workspace_bytes(nnz, n_bags, D, K), dtype=torch.uint8,
-                     device="cuda")
+    size = (B.antdt_embbag_bwd_dedup_min_workspace_bytes if min_workspace
+            else B.antdt_embbag_bwd_dedup_workspace_bytes)(nnz, n_bags, D, K)
+    ws = torch.empty(size, dtype=torch.uint8, device="cuda")
     st = new_status()
     B.antdt_embbag_bwd_dedup(dev(ids), dev(off), F, dev(dY), n_rows, [int(x) for x in wso], uid, wuo,
                              so, occ[:nnz], ug, ws, st)

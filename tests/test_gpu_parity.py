@@ -113,6 +113,39 @@ def test_bwd_dedup_large_multi_chunk_with_hot_rows():
     assert np.diff(want["seg_offsets"]).max() > 20_000
 
 
+def test_bwd_with_the_minimum_workspace_walks_long_tiles():
+    """Up to 2^20 occurrences the recommended workspace buys 16-entry reduction tiles; with the
+    minimum workspace the same call walks 64-entry tiles.  Integer outputs identical, sums within
+    tolerance of the checker either way; one byte less than the minimum is refused."""
+    rng = np.random.default_rng(77)
+    V, D, K, F, S = 20_000, 32, 5, 6, 9000
+    ids, off = random_bags(rng, S * F, V, 9, zipf=1.2)        # ~270k occurrences, long hot runs
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    wso = _wso(rng, K, S)
+    nnz = len(ids)
+    rec = B.antdt_embbag_bwd_dedup_workspace_bytes(nnz, S * F, D, K)
+    least = B.antdt_embbag_bwd_dedup_min_workspace_bytes(nnz, S * F, D, K)
+    assert least < rec
+    big = B.antdt_embbag_bwd_dedup_workspace_bytes(3 << 20, 1000, D, K)
+    assert big == B.antdt_embbag_bwd_dedup_min_workspace_bytes(3 << 20, 1000, D, K)
+    a = G.gpu_bwd(ids, off, F, dY, V, wso)
+    b = G.gpu_bwd(ids, off, F, dY, V, wso, min_workspace=True)
+    want = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+    for got in (a, b):
+        assert got["status"] == 0
+        for k in ("worker_uniq_offsets", "uniq_ids", "seg_offsets", "sorted_occ"):
+            assert np.array_equal(got[k], want[k]), k
+        G.close(got["uniq_grads"], want["uniq_grads"])
+    # below the minimum: refused before any launch
+    cap = max(1, nnz)
+    t = lambda *shape, dt=torch.int32: torch.zeros(*shape, dtype=dt, device="cuda")
+    with pytest.raises(B.AntdtError) as ei:
+        B.antdt_embbag_bwd_dedup(G.dev(ids), G.dev(off), F, G.dev(dY), V, [int(x) for x in wso], t(cap),
+                                 t(K + 1, dt=torch.int64), t(cap + 1, dt=torch.int64), t(nnz),
+                                 t(cap, D, dt=torch.float32), t(least - 256, dt=torch.uint8), G.new_status())
+    assert ei.value.code == B.ERR_WORKSPACE_TOO_SMALL
+
+
 def test_bwd_is_bit_reproducible():
     rng = np.random.default_rng(12)
     V, D, K, F, S = 500, 32, 4, 5, 3000

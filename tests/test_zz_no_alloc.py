@@ -62,7 +62,7 @@ def test_static_scratch_variant_rejects_what_does_not_fit():
     wso = (C.c_int64 * 2)(0, 1)
     n0 = B.antdt_launch_count()
     too_many = 4_000_000           # needs far more than the 24 MiB array at dim 64
-    assert B.antdt_embbag_bwd_dedup_workspace_bytes(too_many, 1, 64, 1) > B.STATIC_SCRATCH_BYTES
+    assert B.antdt_embbag_bwd_dedup_min_workspace_bytes(too_many, 1, 64, 1) > B.STATIC_SCRATCH_BYTES
     rc = L.antdt_embbag_bwd_dedup_static(one, too_many, one, 1, 1, one, 64, 10, 1, wso, one, one, one,
                                          one, one, too_many, None, None)
     assert rc == B.ERR_CAPACITY
