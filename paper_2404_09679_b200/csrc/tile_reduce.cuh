@@ -39,7 +39,7 @@ struct TileArgs {
   int dim;
   int64_t n_host;             // entries (upper bound when n_dev is given)
   const int64_t* n_dev;       // device-side entry count or nullptr
-  int64_t payload_limit;      // payloads >= this are skipped (never dereferenced)
+  int64_t payload_limit;      // rows of the matrix (>= 1); a payload >= this reads the last row
   const int64_t* bounds;      // backward: entry range of every worker [K+1];
                               // aggregation: payload range of every worker [K+1]
   const float* scales;        // backward: 1/b_w [K]; aggregation: weight w_i [K]
@@ -111,30 +111,52 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
   for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
   const uint32_t row_stride = (uint32_t)dim;
 
-  for (int q = 0; q * G < nv; ++q) {
-    int my_row = -1;
+  // Every load of the backward's walk is unconditional: a payload outside the matrix (only possible after
+  // an error that is already flagged) is clamped to the last row, idle lanes of a row whose width
+  // is not a power of two re-read its last vector, and the slots past the data of the last tile
+  // read row 0 - they come after the bit that closes the last run, so their sum is never stored.
+  constexpr int GE = G < TILE ? G : TILE;  // entries a group step covers
+  const uint32_t last_row = (uint32_t)(a.payload_limit - 1);
+  int vi_c[VPL];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) vi_c[k] = min(lg + k * G, nvec - 1);
+  for (int q = 0; q * GE < nv; ++q) {
+    // backward: unconditional loads as described above.  Aggregation (bound by DRAM, and its
+    // weight lookup already fills the register budget): slots without data are marked -1 and
+    // their loads predicated off.
+    int my_row = AGG ? -1 : 0;
     float my_wt = 0.f;
-    if (q * G + lg < nv) {
-      const uint32_t p = __ldg(payload + o_begin + q * G + lg);
-      my_row = ((int64_t)p < a.payload_limit) ? (int)p : -1;  // -1: skipped, contributes nothing
-      if (AGG && my_row >= 0) {
-        int wl = interval_of(s_bounds, K + 1, (int64_t)p);
-        my_wt = s_w[wl > K - 1 ? K - 1 : wl];
+    if (lg < GE && q * GE + lg < nv) {
+      const uint32_t p = __ldg(payload + o_begin + q * GE + lg);
+      if (AGG) {
+        my_row = ((int64_t)p < a.payload_limit) ? (int)p : -1;
+        if (my_row >= 0) {
+          int wl = interval_of(s_bounds, K + 1, (int64_t)p);
+          my_wt = s_w[wl > K - 1 ? K - 1 : wl];
+        }
+      } else {
+        my_row = (int)min(p, last_row);
       }
     }
 #pragma unroll
-    for (int j0 = 0; j0 < G; j0 += U) {
+    for (int j0 = 0; j0 < GE; j0 += U) {
       float4 v[U][VPL];
       float wt[U];
 #pragma unroll
       for (int t = 0; t < U; ++t) {
         const int row = __shfl_sync(gmask, my_row, j0 + t, G);
         wt[t] = AGG ? __shfl_sync(gmask, my_wt, j0 + t, G) : 1.f;
-        const float* rp = rows + (size_t)((uint32_t)(row < 0 ? 0 : row)) * row_stride;
+        if (AGG) {
+          const float* rp = rows + (size_t)((uint32_t)(row < 0 ? 0 : row)) * row_stride;
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-          const int vi = lg + k * G;
-          v[t][k] = (row >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int k = 0; k < VPL; ++k) {
+            const int vi = lg + k * G;
+            v[t][k] = (row >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        } else {
+          const float* rp = rows + (size_t)(uint32_t)row * row_stride;
+#pragma unroll
+          for (int k = 0; k < VPL; ++k) v[t][k] = ldg_f4(rp + 4 * vi_c[k]);
         }
       }
 #pragma unroll
@@ -154,7 +176,7 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
           float sc = 1.f;
           if (started) {
             if (!AGG) {
-              const int rel = q * G + j0 + t;
+              const int rel = q * GE + j0 + t;
               if (rel >= next_w_rel) {  // crossed into a later worker's range
                 const int64_t o = o_begin + rel;
                 while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
@@ -185,7 +207,7 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
         }
       }
     }
-    ends = (G >= 64) ? 0ull : (ends >> (G & 63));
+    ends >>= GE;
   }
   if (open_tail) {
     float* dst = (started ? tail_part : head_part) + (size_t)tile * row_stride;
