@@ -159,6 +159,18 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
           for (int k = 0; k < VPL; ++k) v[t][k] = ldg_f4(rp + 4 * vi_c[k]);
         }
       }
+      if (!AGG && ((ends >> j0) & ((1ull << U) - 1ull)) == 0ull) {
+        // none of these U entries closes a run (the common case inside a hot row): add, no tests
+#pragma unroll
+        for (int t = 0; t < U; ++t) {
+#pragma unroll
+          for (int k = 0; k < VPL; ++k) {
+            acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
+            acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
+          }
+        }
+        continue;
+      }
 #pragma unroll
       for (int t = 0; t < U; ++t) {
 #pragma unroll
