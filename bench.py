@@ -152,8 +152,8 @@ def plan_all(w, n_steps):
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
 # full-size default workload summarised in profiles/; a kernel that has changed since is set to None.
-NCU_TRAFFIC = {4: {"seg_reduce_tiles": 12.95e9, "agg_reduce": 6.80e9, "sparse_adagrad": 9.42e9,
-                   "embbag_fwd": 4.04e9, "radix_scatter": (2.90e9 + 2.34e9 + 2.08e9) / 3}}
+NCU_TRAFFIC = {4: {"seg_reduce_tiles": 13.09e9, "agg_reduce": 6.80e9, "sparse_adagrad": 9.41e9,
+                   "embbag_fwd": 4.04e9, "radix_scatter": (3.29e9 + 2.64e9 + 2.27e9) / 3}}
 
 
 def scaled_workload(w, scale):
