@@ -37,13 +37,23 @@ static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t
 // memory.  bytes % 4 == 0.  Defined in runtime.cu.
 void upload_small(const void* host, size_t bytes, void* dev, cudaStream_t s);
 
+// A d_pooled matrix that is still being copied in when the backward is issued, in n pieces:
+// piece c holds the rows that the occurrences before entry_end[c] (ascending, host array) refer
+// to - in a step these are the workers' sample ranges - and is complete once ready[c] has
+// happened.  Later events imply the earlier ones (one copy stream).
+struct PooledArrival {
+  int n;
+  const int64_t* entry_end;
+  const cudaEvent_t* ready;
+};
+
 int32_t bwd_dedup_impl(const int32_t* row_ids, int64_t nnz, const int64_t* bag_offsets,
                        int64_t n_bags, int32_t bags_per_sample, const float* d_pooled, int32_t dim,
                        int64_t n_rows, int32_t n_workers, const int64_t* worker_sample_offsets,
                        int32_t* uniq_ids, int64_t* worker_uniq_offsets, int64_t* seg_offsets,
                        int32_t* sorted_occ, float* uniq_grads, int64_t out_cap, void* ws,
                        size_t ws_bytes, int32_t* dev_status, void* stream,
-                       cudaEvent_t d_pooled_ready);  // embbag_bwd.cu
+                       const PooledArrival* arrival);  // embbag_bwd.cu
 
 constexpr int kNumSM = 148;  // B200: 2 dies x 74 SMs; grids are sized in multiples of this
 

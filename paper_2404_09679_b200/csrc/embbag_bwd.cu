@@ -122,7 +122,7 @@ int32_t bwd_dedup_impl(
     int32_t bags_per_sample, const float* d_pooled, int32_t dim, int64_t n_rows, int32_t n_workers,
     const int64_t* worker_sample_offsets, int32_t* uniq_ids, int64_t* worker_uniq_offsets,
     int64_t* seg_offsets, int32_t* sorted_occ, float* uniq_grads, int64_t out_cap, void* ws,
-    size_t ws_bytes, int32_t* dev_status, void* stream, cudaEvent_t d_pooled_ready) {
+    size_t ws_bytes, int32_t* dev_status, void* stream, const PooledArrival* arrival) {
   const int K = n_workers;
   if (nnz < 0 || n_bags < 0 || nnz >= (1ll << 31) || n_bags >= (1ll << 31) || n_rows < 1 ||
       n_rows >= (1ll << 31) || dim < 4 || dim > 1024 || dim % 4 || K < 1 || K > kMaxSegments ||
@@ -177,8 +177,6 @@ int32_t bwd_dedup_impl(
   segsort_runs(keys_a, nnz, uniq_ids, seg_offsets, worker_uniq_offsets, nullptr, out_cap,
                (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), tile_len, sort_ws,
                L.sort, dev_status, s);
-  if (d_pooled_ready && cudaStreamWaitEvent(s, d_pooled_ready, 0) != cudaSuccess)
-    return ANTDT_ERR_CUDA;
   if (nnz > 0) {
     TileArgs t;
     t.payload = occ_out;
@@ -197,7 +195,31 @@ int32_t bwd_dedup_impl(
     t.out = uniq_grads;
     t.head_part = (float*)(w8 + L.head_part);
     t.tail_part = (float*)(w8 + L.tail_part);
-    launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+    if (!arrival || arrival->n < 1) {
+      launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+    } else {
+      // d_pooled is arriving piece by piece: a tile is walked as soon as the piece that holds
+      // its last entry is there (the sort and the run detection above needed the ids only)
+      const int64_t n_tiles = (nnz + tile_len - 1) / tile_len;
+      int64_t done = 0;  // tiles issued so far
+      t.fixup = false;
+      for (int c = 0; c < arrival->n; ++c) {
+        if (cudaStreamWaitEvent(s, arrival->ready[c], 0) != cudaSuccess) return ANTDT_ERR_CUDA;
+        int64_t upto = n_tiles;  // the last piece takes every remaining tile
+        if (c + 1 < arrival->n) {
+          const int64_t e = arrival->entry_end[c];
+          upto = e <= 0 ? 0 : (e >= nnz ? n_tiles : e / tile_len);  // tiles that end before entry e
+        }
+        if (upto <= done) continue;
+        t.tile_begin = done;
+        t.tile_end = upto;
+        launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+        done = upto;
+      }
+      t.walk = false;
+      t.fixup = true;
+      launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+    }
   }
   return cuda_ok();
 }

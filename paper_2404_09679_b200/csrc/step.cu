@@ -10,10 +10,12 @@
 
 namespace {
 // Side streams and events of the host-buffer step, created on first use for each device.
+constexpr int kMaxPieces = 16;  // the d_pooled copy is cut into at most this many pieces
 struct StepStreams {
   bool ready = false;
   cudaStream_t in = nullptr, out = nullptr;
-  cudaEvent_t start, ids, dy, dense, fwd, done, outdone;
+  cudaEvent_t start, ids, dense, fwd, done, outdone;
+  cudaEvent_t piece[kMaxPieces];
 };
 StepStreams g_ss[64];
 std::mutex g_ss_mu;
@@ -26,9 +28,11 @@ StepStreams* step_streams() {
   if (!ss.ready) {
     if (cudaStreamCreateWithFlags(&ss.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&ss.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    cudaEvent_t* ev[] = {&ss.start, &ss.ids, &ss.dy, &ss.dense, &ss.fwd, &ss.done, &ss.outdone};
+    cudaEvent_t* ev[] = {&ss.start, &ss.ids, &ss.dense, &ss.fwd, &ss.done, &ss.outdone};
     for (cudaEvent_t* e : ev)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (cudaEvent_t& e : ss.piece)
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     ss.ready = true;
   }
   return &ss;
@@ -63,10 +67,41 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
     CK(cudaMemcpyAsync(d->d_row_ids, d->h_row_ids, 4 * (size_t)d->nnz, cudaMemcpyHostToDevice,
                        ss->in));
   CK(cudaEventRecord(ss->ids, ss->in));
-  if (d->n_bags > 0)
-    CK(cudaMemcpyAsync(d->d_d_pooled, d->h_d_pooled, 4 * (size_t)d->n_bags * D,
-                       cudaMemcpyHostToDevice, ss->in));
-  CK(cudaEventRecord(ss->dy, ss->in));
+  // d_pooled is the largest input and the backward's reduction is the first to read it: it is
+  // copied in pieces of whole workers, each with its own event, so that the reduction of a
+  // worker's occurrences starts when that worker's rows are there (only the last piece's
+  // reduction is left once the copy ends).  Small inputs travel as one piece.
+  int n_pieces = 0;
+  int64_t piece_entry_end[kMaxPieces];
+  if (d->n_bags > 0) {
+    const int K = d->n_workers;
+    const int64_t F = d->bags_per_sample;
+    const size_t row_bytes = 4 * D;
+    const bool cut = K > 1 && F > 0 && d->worker_sample_offsets &&
+                     (size_t)d->n_bags * row_bytes >= ((size_t)8 << 20);
+    const int want = cut ? (K < kMaxPieces ? K : kMaxPieces) : 1;
+    int64_t bag0 = 0;
+    int w0 = 0;
+    for (int c = 0; c < want; ++c) {
+      // workers [w0, w1): an equal share of the workers per piece, the last piece takes the rest
+      const int w1 = c + 1 == want ? K : (int)(((int64_t)(c + 1) * K) / want);
+      int64_t bag1 = c + 1 == want ? d->n_bags : d->worker_sample_offsets[w1] * F;
+      if (bag1 < bag0) bag1 = bag0;
+      if (bag1 > d->n_bags) bag1 = d->n_bags;
+      if (bag1 > bag0)
+        CK(cudaMemcpyAsync(d->d_d_pooled + (size_t)bag0 * D, d->h_d_pooled + (size_t)bag0 * D,
+                           (size_t)(bag1 - bag0) * row_bytes, cudaMemcpyHostToDevice, ss->in));
+      CK(cudaEventRecord(ss->piece[c], ss->in));
+      int64_t e = d->h_bag_offsets[bag1];  // occurrences before the piece's end (host copy)
+      if (e < 0) e = 0;
+      if (e > d->nnz) e = d->nnz;
+      piece_entry_end[c] = e;
+      bag0 = bag1;
+      w0 = w1;
+    }
+    (void)w0;
+    n_pieces = want;
+  }
   if (dense)
     CK(cudaMemcpyAsync(d->d_dense_grads, d->h_dense_grads,
                        4 * (size_t)d->n_workers * (size_t)d->dense_n, cudaMemcpyHostToDevice,
@@ -84,11 +119,12 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
   if (d->h_pooled && d->n_bags > 0)
     CK(cudaMemcpyAsync(d->h_pooled, d->d_pooled_out, 4 * (size_t)d->n_bags * D,
                        cudaMemcpyDeviceToHost, ss->out));
+  antdt::PooledArrival arrival{n_pieces, piece_entry_end, ss->piece};
   rc = antdt::bwd_dedup_impl(d->d_row_ids, d->nnz, d->d_bag_offsets, d->n_bags, d->bags_per_sample,
                               d->d_d_pooled, d->dim, d->n_rows, d->n_workers,
                               d->worker_sample_offsets, d->d_uniq_ids, d->d_worker_uniq_offsets,
                               d->d_seg_offsets, d->d_sorted_occ, d->d_uniq_grads, d->uniq_cap, d->ws,
-                              d->ws_bytes, d->d_status, stream, ss->dy);
+                              d->ws_bytes, d->d_status, stream, n_pieces > 0 ? &arrival : nullptr);
   if (rc != ANTDT_OK) return rc;
   CK(cudaStreamWaitEvent(s, ss->dense, 0));
   antdt_sparse_part sp;

@@ -48,6 +48,12 @@ struct TileArgs {
   float* out;                 // [out_cap, dim]
   float* head_part;           // [n_tiles, dim]
   float* tail_part;           // [n_tiles, dim]
+  // Which part of the work a launch_tile_reduce call issues (defaults: everything).  A caller
+  // whose `rows` arrive in pieces walks the tiles piece by piece and runs the fix-up last.
+  int64_t tile_begin = 0;     // first tile of the walk
+  int64_t tile_end = -1;      // one past its last tile; -1: to the end
+  bool walk = true;           // issue the tile walk over [tile_begin, tile_end)
+  bool fixup = true;          // issue the fix-up pass (over all tiles)
 };
 
 // The hot pointers are separate __restrict__ parameters (not read through the struct) so that
@@ -67,9 +73,9 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
   __syncthreads();
   const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
   const int lg = threadIdx.x & (G - 1);
-  const int64_t tile = (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
+  const int64_t tile = a.tile_begin + (int64_t)blockIdx.x * (kRedThreads / G) + threadIdx.x / G;
   const int64_t o_begin = tile * TILE;
-  if (o_begin >= n) return;
+  if (tile >= a.tile_end || o_begin >= n) return;
   const int nv = (int)min((int64_t)TILE, n - o_begin);  // entries in this tile
   const unsigned gmask = group_mask<G>();
   const int dim = a.dim;
@@ -319,16 +325,23 @@ tile_fixup_kernel(const TileArgs a) {
 }
 
 template <int G, int VPL, bool AGG, int TILE>
-void launch_tile_reduce_t(const TileArgs& a, const char* name_tiles, const char* name_fixup,
+void launch_tile_reduce_t(const TileArgs& a_in, const char* name_tiles, const char* name_fixup,
                           cudaStream_t s) {
-  const int64_t n_tiles = (a.n_host + TILE - 1) / TILE;
+  const int64_t n_tiles = (a_in.n_host + TILE - 1) / TILE;
   const int64_t tpb = kRedThreads / G;
-  const unsigned grid = (unsigned)((n_tiles + tpb - 1) / tpb);
-  if (grid == 0) return;
+  TileArgs a = a_in;
+  if (a.tile_begin < 0) a.tile_begin = 0;
+  if (a.tile_end < 0 || a.tile_end > n_tiles) a.tile_end = n_tiles;
   const size_t smem = 8 * ((size_t)a.K + 1) + (AGG ? 4 * (size_t)a.K : 0);
-  ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, smem, s, a,
-               a.payload, a.head_bits, a.tile_first, a.rows, a.out, a.head_part, a.tail_part);
-  ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, 0, s, a);
+  if (a.walk && a.tile_end > a.tile_begin) {
+    const unsigned grid = (unsigned)((a.tile_end - a.tile_begin + tpb - 1) / tpb);
+    ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, smem, s, a,
+                 a.payload, a.head_bits, a.tile_first, a.rows, a.out, a.head_part, a.tail_part);
+  }
+  if (a.fixup && n_tiles > 0) {
+    const unsigned grid = (unsigned)((n_tiles + tpb - 1) / tpb);
+    ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, 0, s, a);
+  }
 }
 
 template <int G, int VPL, bool AGG>
