@@ -2,9 +2,12 @@
 """Benchmark of the BSP sparse-ranking step: training samples/s per step on B200.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+                  [--launch auto|graph|stream]
 
 One step = planner call + embbag_fwd + embbag_bwd_dedup + weighted_aggregate + sparse_opt_update
-over one batch of seeded synthetic input.  `value` is measured with the batch resident in HBM;
+over one batch of seeded synthetic input.  `value` is measured with the batch resident in HBM
+(plain launches through antdt_bsp_step_device; the launch-bound configurations 1 and 2 as one CUDA
+graph per step through antdt_bsp_step_graph);
 `e2e` goes through antdt_bsp_step_host with page-locked HOST buffers (copies inside the timed
 region).  The path does not shard (one GPU holds the whole table): with N > 1 every rank runs an
 independent replica and the job value is the sum of the replicas' samples over the slowest time.
@@ -152,8 +155,8 @@ def plan_all(w, n_steps):
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
 # full-size default workload summarised in profiles/; a kernel that has changed since is set to None.
-NCU_TRAFFIC = {4: {"seg_reduce_tiles": 13.09e9, "agg_reduce": 6.80e9, "sparse_adagrad": 9.41e9,
-                   "embbag_fwd": 4.04e9, "radix_scatter": (3.29e9 + 2.64e9 + 2.27e9) / 3}}
+NCU_TRAFFIC = {4: {"seg_reduce_tiles": 12.80e9, "agg_reduce": 6.77e9, "sparse_adagrad": 9.41e9,
+                   "embbag_fwd": 4.04e9, "radix_scatter": 2.44e9}}
 
 
 def scaled_workload(w, scale):

@@ -11,11 +11,13 @@
 // piece and the following head pieces in tile order.  Every sum has a fixed order: no
 // floating-point atomics, bit-reproducible.
 //
-// The walk is issue-bound once the gathered rows sit in L2, so it is built to cost few
+// The walk is issue-bound once the gathered rows sit in L1/L2, so it is built to cost few
 // instructions per entry: the tile's run ends are one 64-bit mask consumed with constant
-// shifts, the payloads of G entries live in one register per lane and are broadcast by shuffle,
-// kRedUnroll row loads are in flight before the first add, and in the backward the worker (for
-// the 1/b_w scale) is only re-resolved when the walk crosses a worker boundary.
+// shifts and tested once per kRedUnroll entries (inside a hot row nothing closes, and the
+// entries are only added), the payloads of G entries live in one register per lane and are
+// broadcast by shuffle, kRedUnroll row loads are in flight before the first add, the backward's
+// loads are unconditional (clamped indices instead of predicates), and the worker (for the 1/b_w
+// scale) is only re-resolved when the walk crosses a worker boundary.
 #pragma once
 #include "common.cuh"
 
