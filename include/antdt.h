@@ -81,7 +81,7 @@ typedef struct antdt_dds antdt_dds; /* opaque; host memory owned by the library 
 /* Section V-C.1.  Splits n_samples samples into ceil(n_samples / (global_batch *
  * batches_per_shard)) shards of global_batch*batches_per_shard consecutive samples (the last
  * one shorter), all in state TODO, and queues them in index order; shuffle_seed != 0 permutes
- * the queue with a seeded Fisher-Yates (the "shuffle between shards" of the Shard Shuffler).
+ * the queue with a seeded Fisher-Yates (the Shard Shuffler's permutation of whole shards).
  * *out receives the handle; release it with antdt_dds_destroy.
  * INVALID_ARG: NULL out, n_samples < 1, global_batch < 1, batches_per_shard < 1,
  * n_workers outside [1, 1024]. */
@@ -262,8 +262,8 @@ int32_t antdt_embbag_bwd_dedup_static(const int32_t* row_ids, int64_t nnz,
                                       int32_t* sorted_occ, float* uniq_grads, int64_t out_cap,
                                       int32_t* dev_status, void* stream);
 
-/* Server aggregation (Section II: "the servers aggregate the local gradients from all
- * workers"; the global batch is fixed, Eq. 1's last constraint).  Workers push MEAN gradients
+/* Server aggregation (Section II: the servers combine the local gradients of all workers into
+ * one; the global batch is fixed, Eq. 1's last constraint).  Workers push MEAN gradients
  * over unequal local batches, so the aggregate that equals the mean over the global batch is
  *     G = sum_i (b_i / sum_j b_j) * G_i.
  * Sparse part: agg_ids = ascending union of the workers' row lists, a worker that does not
@@ -307,7 +307,7 @@ int32_t antdt_weighted_aggregate_backup(const antdt_sparse_part* sp, const antdt
                                         int32_t n_workers, void* ws, size_t ws_bytes,
                                         int32_t* dev_status, void* stream);
 
-/* Server update (Section II: the servers "update the parameters"), on the rows in ids only;
+/* Server update (Section II: the servers then apply the gradient to the parameters), on the rows in ids only;
  * every other row of table and state is left bit-identical.
  *   Adagrad: state0 += g*g;  w -= lr * g / (sqrt(state0) + eps)
  *   Adam:    state0 = b1*state0 + (1-b1)*g;  state1 = b2*state1 + (1-b2)*g*g;

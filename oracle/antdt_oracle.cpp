@@ -14,7 +14,7 @@
 // Where the paper fixes the computation, the passage is cited beside the function; the
 // embedding-bag, dedup, weighting and optimizer definitions are the textbook ones the paper
 // leaves to its training substrate (Section II only says workers compute local gradients on
-// B_i and servers "aggregate the local gradients ... and update the parameters").
+// B_i and that the servers combine them and apply the result to the parameters).
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
