@@ -35,6 +35,19 @@ def test_checker_transient_but_not_persistent():
     assert oracle.batch_sizes(v, 3, 576).tolist() == [256, 256, 64]
 
 
+def test_lambda_test_flags_a_worker_exactly_at_the_threshold():
+    # Section VI-A step 3 prints the test with ">=".  Batch-processing times 1, 1, 1, 3 (all exact
+    # in binary): mean 1.5, lambda 2 -> threshold exactly 3.0, so worker 3 IS a straggler; a strict
+    # comparison would let it pass.  One ulp below the threshold it is not.
+    rep = [(w, 128, 3.0 if w == 3 else 1.0) for _ in range(4) for w in range(4)]
+    v, t, p, a = oracle.ctl_decide(rep, 4, 2, 4, 2.0)
+    assert t.tolist() == [0, 0, 0, 1] and p.tolist() == [0, 0, 0, 1] and a == 2
+    below = float(np.nextafter(3.0, 0.0))
+    rep = [(w, 128, below if w == 3 else 1.0) for _ in range(4) for w in range(4)]
+    v, t, p, a = oracle.ctl_decide(rep, 4, 2, 4, 2.0)
+    assert t.sum() == 0 and p.sum() == 0 and a == 0
+
+
 def test_throughput_is_mean_of_per_report_rates():
     rep = [(0, 100, 1.0), (0, 300, 2.0), (1, 100, 1.0), (1, 100, 1.0)]
     v, _, _, _ = oracle.ctl_decide(rep, 2, 5, 5, 1.5)

@@ -198,6 +198,24 @@ def test_adagrad_closed_form_constant_gradient():
     assert np.all(W[mask] == 0.5) and np.all(acc[mask] == 0)
 
 
+def test_adagrad_eps_sits_outside_the_square_root():
+    # One step from a zero accumulator with eps as large as |g|: acc = g^2, so the element moves by
+    # -lr g / (|g| + eps) = -lr/2 exactly in binary arithmetic.  With eps under the root the move
+    # would be -lr g / sqrt(g^2 + eps) = -lr / sqrt(1 + 2^10) ~ -0.0312 lr: a factor of 16 away.
+    lr, eps = 0.5, 2.0 ** -10
+    g = np.array([[2.0 ** -10, -(2.0 ** -10), 2.0 ** -10, -(2.0 ** -10)]], np.float32)
+    W = np.zeros((2, 4), np.float32)
+    acc = np.zeros((2, 4), np.float32)
+    oracle.sparse_opt_update(W, np.array([1], np.int32), g, "adagrad", lr, eps, 0, 0, 1, acc)
+    assert np.array_equal(acc[1], np.full(4, 2.0 ** -20, np.float32))
+    assert np.array_equal(W[1], np.array([-0.25, 0.25, -0.25, 0.25], np.float32))
+    assert np.all(W[0] == 0) and np.all(acc[0] == 0)
+    # second step, same gradient: acc = 2 g^2, move = -lr g / (sqrt(2)|g| + eps) = -lr/(sqrt 2 + 1)
+    oracle.sparse_opt_update(W, np.array([1], np.int32), g, "adagrad", lr, eps, 0, 0, 2, acc)
+    want = -np.sign(g[0].astype(np.float64)) * (0.25 + 0.5 / (np.sqrt(2.0) + 1.0))
+    assert np.allclose(W[1], want, rtol=1e-6)
+
+
 def test_zero_gradient_row_is_unchanged():
     W = np.full((3, 4), 0.3, np.float32)
     acc = np.full((3, 4), 2.0, np.float32)
@@ -275,6 +293,21 @@ def test_rowwise_adagrad_closed_form_constant_gradient():
     assert np.allclose(W[2], want, rtol=1e-6)
     mask = np.arange(V) != 2
     assert np.all(W[mask] == np.float32(-0.25)) and np.all(acc[mask] == 0)
+
+
+def test_rowwise_adagrad_eps_sits_outside_the_square_root():
+    # |g_c| = 2^-10 for every element, eps = 2^-10, zero state: the row's mean square is 2^-20, its
+    # root 2^-10 = eps, so every element moves by -lr sign(g)/2 exactly.  eps under the root would
+    # give -lr sign(g) 2^-10 / sqrt(2^-20 + 2^-10), 16 times smaller.
+    lr, eps = 0.5, 2.0 ** -10
+    s = np.array([1, -1, -1, 1, 1, 1, -1, 1], np.float64)
+    g = (s * 2.0 ** -10).astype(np.float32)[None, :]
+    W = np.zeros((3, 8), np.float32)
+    acc = np.zeros(3, np.float32)
+    oracle.sparse_rowwise_adagrad(W, np.array([2], np.int32), g, lr, eps, acc)
+    assert acc[2] == np.float32(2.0 ** -20) and acc[0] == 0 and acc[1] == 0
+    assert np.array_equal(W[2], (-0.25 * s).astype(np.float32))
+    assert np.all(W[:2] == 0)
 
 
 def test_rowwise_adagrad_equals_elementwise_when_magnitudes_are_equal():
