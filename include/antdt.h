@@ -108,8 +108,9 @@ int32_t antdt_batch_sizes(const double* speeds, int32_t n_workers, int64_t globa
  * batch_sizes[i] samples from the shard it currently holds; a worker whose shard runs out
  * fetches the TODO shard at the head of the queue (it becomes DOING and cannot go to anyone
  * else) and goes on, so a worker's step is a short list of ranges.  A shard whose last sample
- * was served is DONE when the call returns (the step's gradients count as pushed).  When the
- * queue is empty a worker's step is short: counts[i] < batch_sizes[i].
+ * was served is DONE when the call returns (the step's gradients count as pushed) unless
+ * antdt_dds_requeue_worker reports, before the next antdt_shard_plan, that the worker's push
+ * failed.  When the queue is empty a worker's step is short: counts[i] < batch_sizes[i].
  *   batch_sizes   host out [K]   planned sizes, sum = global_batch
  *   range_offsets host out [K+1] CSR offsets into ranges
  *   ranges        host out [ranges_cap]
@@ -120,9 +121,13 @@ int32_t antdt_shard_plan(antdt_dds* dds, const double* speeds, int32_t rule, int
                          int64_t* batch_sizes, int64_t* range_offsets, antdt_range* ranges,
                          int64_t ranges_cap, int64_t* counts);
 
-/* Section V-C.3, last paragraph: the shard a lost worker (BACKUP_WORKERS drop, KILL_RESTART)
- * was DOING goes back to TODO at the END of the queue and will be served again in full
- * (at-least-once).  No-op if the worker holds no shard. */
+/* Section V-C.3, last paragraph: the shards of a lost worker (BACKUP_WORKERS drop,
+ * KILL_RESTART) go back to TODO at the END of the queue and will be served again in full
+ * (at-least-once): first every shard whose last sample the latest antdt_shard_plan call served
+ * to this worker (a shard is DONE only once its gradients are pushed, and this worker's were
+ * not), in the order it finished them, then the shard it is DOING.  Call it between the plan
+ * call whose gradients were lost and the next one; later, only the DOING shard is returned.
+ * No-op if the worker holds and finished nothing. */
 int32_t antdt_dds_requeue_worker(antdt_dds* dds, int32_t worker);
 
 /* Shard bookkeeping used by the integrity checks (Section VII-D: #DONE = ceil(N/(B*M))). */

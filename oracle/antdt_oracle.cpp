@@ -21,6 +21,7 @@
 #include <cstring>
 #include <deque>
 #include <limits>
+#include <utility>
 #include <vector>
 
 namespace {
@@ -135,13 +136,16 @@ int batch_sizes(const double* v, int n, i64 B, int rule, i64 minb, i64* b) {
 // ---------------------------------------------------------------------------------------
 // Stateful Dynamic Data Sharding, Section V-C.
 // ---------------------------------------------------------------------------------------
-struct Shard { i64 start, len; int state; int owner; };
+// done_by / done_plan / done_seq: who served the shard's last sample, in which plan call, and
+// the position of that event among all such events (a global counter).
+struct Shard { i64 start, len; int state; int owner; int done_by; i64 done_plan, done_seq; };
 
 struct Dds {
   i64 N, B; int M, K;
   std::vector<Shard> shards;
   std::deque<i64> queue;         // TODO shards, head = next to hand out
   std::vector<i64> held, used;   // per worker: shard it is DOING (-1 none), samples consumed
+  i64 plans = 0, seq = 0;        // committed plan calls; completion events so far
 };
 
 uint64_t sm64_next(uint64_t& s) {
@@ -218,6 +222,7 @@ void* orc_dds_create(i64 N, i64 B, int M, int K, uint64_t shuffle_seed) {
     s.start = j * per;
     s.len = std::min(per, N - s.start);
     s.state = 0; s.owner = -1;
+    s.done_by = -1; s.done_plan = -1; s.done_seq = -1;
     d->shards.push_back(s);
   }
   std::vector<i64> order(n_sh);
@@ -252,7 +257,9 @@ void orc_dds_shard_info(void* h, i64 j, int* state, int* owner, i64* start, i64*
 // One BSP step of the service.  Workers are served in ascending index; a worker keeps the
 // shard it is DOING until it has consumed all of it (Section V-C.2: it cannot fetch a new one
 // before), then takes the queue head (TODO -> DOING).  A shard whose last sample was served is
-// DONE once the step's gradients are pushed, i.e. when this call returns (Section V-C.3).
+// DONE once the step's gradients are pushed (Section V-C.3): it is marked DONE when this call
+// returns, and orc_dds_requeue takes the mark back if the push turns out to have failed before
+// the next call.
 // ranges: int64 pairs (start, len), CSR by worker through range_offsets.
 int orc_dds_plan(void* h, const double* speeds, int rule, i64 min_batch, i64* bsz,
                  i64* range_offsets, i64* ranges, i64 cap, i64* counts) {
@@ -260,6 +267,7 @@ int orc_dds_plan(void* h, const double* speeds, int rule, i64 min_batch, i64* bs
   int rc = batch_sizes(speeds, d->K, d->B, rule, min_batch, bsz);
   if (rc != OK) return rc;
   Dds trial = *d;  // work on a copy; commit only if the ranges fit
+  trial.plans += 1;
   std::vector<i64> out;
   i64 total = 0;
   for (int i = 0; i < trial.K; ++i) {
@@ -284,6 +292,9 @@ int orc_dds_plan(void* h, const double* speeds, int rule, i64 min_batch, i64* bs
       if (trial.used[i] == s.len) {
         s.state = 2;
         s.owner = -1;
+        s.done_by = i;
+        s.done_plan = trial.plans;
+        s.done_seq = trial.seq++;
         trial.held[i] = -1;
         trial.used[i] = 0;
       }
@@ -299,10 +310,26 @@ int orc_dds_plan(void* h, const double* speeds, int rule, i64 min_batch, i64* bs
   return OK;
 }
 
-// Section V-C.3: a lost worker's DOING shard returns to TODO at the END of the queue.
+// Section V-C.3: the shards of a worker whose push failed go back to TODO at the END of the
+// queue: those whose last sample it was served in the latest plan call (their gradients never
+// arrived, so they are not DONE after all), oldest completion first, then the one it is DOING.
 int orc_dds_requeue(void* h, int worker) {
   Dds* d = (Dds*)h;
   if (worker < 0 || worker >= d->K) return E_ARG;
+  std::vector<std::pair<i64, i64>> undone;  // (completion order, shard)
+  for (size_t j = 0; j < d->shards.size(); ++j) {
+    const Shard& s = d->shards[j];
+    if (s.state == 2 && s.done_by == worker && s.done_plan == d->plans)
+      undone.push_back(std::make_pair(s.done_seq, (i64)j));
+  }
+  std::sort(undone.begin(), undone.end());
+  for (const auto& e : undone) {
+    Shard& s = d->shards[e.second];
+    s.state = 0;
+    s.owner = -1;
+    s.done_by = -1;
+    d->queue.push_back(e.second);
+  }
   i64 j = d->held[worker];
   if (j < 0) return OK;
   d->shards[j].state = 0;

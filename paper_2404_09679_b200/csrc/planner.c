@@ -7,6 +7,11 @@
  * n_shards + #requeues entries); every worker has the shard it holds and how much of it is
  * consumed.  A step is planned in two sweeps over the same routine: a dry run on scratch
  * copies of the small per-worker state that only counts ranges, then the committing run.
+ *
+ * A shard becomes DONE only once the gradients computed on its last samples have been pushed
+ * (Section V-C.3).  The planner learns of a failed push through antdt_dds_requeue_worker, so the
+ * shards a worker finished in the latest plan call stay on that worker's short "finished" list
+ * until the next plan call: a requeue in between takes them back together with the DOING shard.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -15,6 +20,10 @@
 #include "antdt.h"
 
 #define MAX_WORKERS 1024
+/* Shards one worker can finish in one step: the one it holds, then only shards no longer than
+ * what is left of its batch (<= B), i.e. the short last shard of the dataset, or a whole shard
+ * when B*M == B_i.  Two at most; the list has room for four, a fifth would simply stay DONE. */
+#define MAX_FINISHED 4
 #define DDS_MAGIC 0x53444454414E41ull /* "ANATDDS" */
 
 struct antdt_dds {
@@ -30,6 +39,8 @@ struct antdt_dds {
   int64_t q_head, q_tail, q_cap;
   int64_t* held;  /* [K] shard a worker is DOING, -1 if none */
   int64_t* used;  /* [K] samples of it already served */
+  int64_t* fin;   /* [K][MAX_FINISHED] shards the worker finished in the latest plan call */
+  int32_t* n_fin; /* [K] how many */
 };
 
 /* ---- splitmix64 stream (Steele, Lea, Flood 2014) for the shard shuffle --------------- */
@@ -166,7 +177,7 @@ int32_t antdt_batch_sizes(const double* speeds, int32_t n_workers, int64_t globa
 static void dds_free(antdt_dds* d) {
   if (!d) return;
   free(d->shard_start); free(d->shard_len); free(d->shard_state); free(d->shard_owner);
-  free(d->queue); free(d->held); free(d->used);
+  free(d->queue); free(d->held); free(d->used); free(d->fin); free(d->n_fin);
   free(d);
 }
 
@@ -181,11 +192,13 @@ static antdt_dds* dds_alloc(int64_t n_shards, int32_t K, int64_t q_cap) {
   d->queue = (int64_t*)malloc(8 * (size_t)q_cap);
   d->held = (int64_t*)malloc(8 * (size_t)K);
   d->used = (int64_t*)malloc(8 * (size_t)K);
+  d->fin = (int64_t*)malloc(8 * (size_t)K * MAX_FINISHED);
+  d->n_fin = (int32_t*)calloc((size_t)K, 4);
   d->q_cap = q_cap;
   d->n_shards = n_shards;
   d->n_workers = K;
   if (!d->shard_start || !d->shard_len || !d->shard_state || !d->shard_owner || !d->queue ||
-      !d->held || !d->used) {
+      !d->held || !d->used || !d->fin || !d->n_fin) {
     dds_free(d);
     return NULL;
   }
@@ -234,7 +247,7 @@ static int64_t serve(antdt_dds* d, const int64_t* bsz, int commit, int64_t* rang
   int64_t n_ranges = 0, q_head = d->q_head, total = 0;
   for (int32_t i = 0; i < d->n_workers; ++i) {
     int64_t held = d->held[i], used = d->used[i], need = bsz[i];
-    if (commit) range_offsets[i] = n_ranges;
+    if (commit) { range_offsets[i] = n_ranges; d->n_fin[i] = 0; }
     while (need > 0) {
       if (held < 0) {
         if (q_head == d->q_tail) break; /* nothing left to fetch: short batch */
@@ -248,8 +261,12 @@ static int64_t serve(antdt_dds* d, const int64_t* bsz, int commit, int64_t* rang
       ++n_ranges;
       used += take;
       need -= take;
-      if (used == d->shard_len[held]) { /* consumed: DONE once this step's push succeeds */
-        if (commit) { d->shard_state[held] = ANTDT_SHARD_DONE; d->shard_owner[held] = -1; }
+      if (used == d->shard_len[held]) { /* consumed: DONE, unless this step's push fails */
+        if (commit) {
+          d->shard_state[held] = ANTDT_SHARD_DONE;
+          d->shard_owner[held] = -1;
+          if (d->n_fin[i] < MAX_FINISHED) d->fin[(size_t)i * MAX_FINISHED + d->n_fin[i]++] = held;
+        }
         held = -1;
         used = 0;
       }
@@ -283,10 +300,8 @@ int32_t antdt_shard_plan(antdt_dds* dds, const double* speeds, int32_t rule, int
   return ANTDT_OK;
 }
 
-int32_t antdt_dds_requeue_worker(antdt_dds* dds, int32_t worker) {
-  if (!dds || worker < 0 || worker >= dds->n_workers) return ANTDT_ERR_INVALID_ARG;
-  int64_t j = dds->held[worker];
-  if (j < 0) return ANTDT_OK;
+/* Appends shard j to the back of the queue (Section V-C.3) as TODO. */
+static int32_t queue_push_back(antdt_dds* dds, int64_t j) {
   if (dds->q_tail == dds->q_cap) { /* compact the consumed prefix, grow if still full */
     int64_t live = dds->q_tail - dds->q_head;
     memmove(dds->queue, dds->queue + dds->q_head, 8 * (size_t)live);
@@ -300,9 +315,25 @@ int32_t antdt_dds_requeue_worker(antdt_dds* dds, int32_t worker) {
       dds->q_cap = cap;
     }
   }
-  dds->queue[dds->q_tail++] = j; /* back of the queue (Section V-C.3) */
+  dds->queue[dds->q_tail++] = j;
   dds->shard_state[j] = ANTDT_SHARD_TODO;
   dds->shard_owner[j] = -1;
+  return ANTDT_OK;
+}
+
+int32_t antdt_dds_requeue_worker(antdt_dds* dds, int32_t worker) {
+  if (!dds || worker < 0 || worker >= dds->n_workers) return ANTDT_ERR_INVALID_ARG;
+  /* the shards it finished in the latest plan call first, in the order it finished them ... */
+  for (int32_t k = 0; k < dds->n_fin[worker]; ++k) {
+    int32_t rc = queue_push_back(dds, dds->fin[(size_t)worker * MAX_FINISHED + k]);
+    if (rc != ANTDT_OK) return rc;
+  }
+  dds->n_fin[worker] = 0;
+  /* ... then the one it is DOING */
+  int64_t j = dds->held[worker];
+  if (j < 0) return ANTDT_OK;
+  int32_t rc = queue_push_back(dds, j);
+  if (rc != ANTDT_OK) return rc;
   dds->held[worker] = -1;
   dds->used[worker] = 0;
   return ANTDT_OK;
@@ -330,17 +361,20 @@ int32_t antdt_dds_shard_info(const antdt_dds* dds, int64_t shard, int32_t* state
 }
 
 /* ---- image: header of 10 int64, then state[n_shards] owner[n_shards] (as int64 each),
- * queue[live], held[K], used[K].  Shard (start, len) are recomputed from the header. ---- */
+ * queue[live], held[K], used[K], n_fin[K], fin[K][MAX_FINISHED].  Shard (start, len) are
+ * recomputed from the header. ---- */
+#define DDS_IMAGE_VERSION 2
 int32_t antdt_dds_save(const antdt_dds* dds, void* buf, size_t cap, size_t* used) {
   if (!dds || !used) return ANTDT_ERR_INVALID_ARG;
   int64_t live = dds->q_tail - dds->q_head;
-  size_t words = 10 + 2 * (size_t)dds->n_shards + (size_t)live + 2 * (size_t)dds->n_workers;
+  size_t words = 10 + 2 * (size_t)dds->n_shards + (size_t)live +
+                 (3 + MAX_FINISHED) * (size_t)dds->n_workers;
   *used = words * 8;
   if (!buf) return ANTDT_OK;
   if (cap < *used) return ANTDT_ERR_CAPACITY;
   int64_t* w = (int64_t*)buf;
   size_t k = 0;
-  w[k++] = (int64_t)DDS_MAGIC; w[k++] = 1;
+  w[k++] = (int64_t)DDS_MAGIC; w[k++] = DDS_IMAGE_VERSION;
   w[k++] = dds->n_samples; w[k++] = dds->global_batch; w[k++] = dds->batches_per_shard;
   w[k++] = dds->n_workers; w[k++] = (int64_t)dds->shuffle_seed; w[k++] = dds->n_shards;
   w[k++] = live; w[k++] = 0;
@@ -349,19 +383,23 @@ int32_t antdt_dds_save(const antdt_dds* dds, void* buf, size_t cap, size_t* used
   for (int64_t j = dds->q_head; j < dds->q_tail; ++j) w[k++] = dds->queue[j];
   for (int32_t i = 0; i < dds->n_workers; ++i) w[k++] = dds->held[i];
   for (int32_t i = 0; i < dds->n_workers; ++i) w[k++] = dds->used[i];
+  for (int32_t i = 0; i < dds->n_workers; ++i) w[k++] = dds->n_fin[i];
+  for (int32_t i = 0; i < dds->n_workers; ++i)
+    for (int32_t f = 0; f < MAX_FINISHED; ++f)
+      w[k++] = f < dds->n_fin[i] ? dds->fin[(size_t)i * MAX_FINISHED + f] : -1;
   return ANTDT_OK;
 }
 
 int32_t antdt_dds_load(antdt_dds** out, const void* buf, size_t len) {
   if (!out || !buf || len < 80 || len % 8) return ANTDT_ERR_INVALID_ARG;
   const int64_t* w = (const int64_t*)buf;
-  if (w[0] != (int64_t)DDS_MAGIC || w[1] != 1) return ANTDT_ERR_INVALID_ARG;
+  if (w[0] != (int64_t)DDS_MAGIC || w[1] != DDS_IMAGE_VERSION) return ANTDT_ERR_INVALID_ARG;
   int64_t N = w[2], B = w[3], M = w[4], K = w[5], n_shards = w[7], live = w[8];
   if (N < 1 || B < 1 || M < 1 || K < 1 || K > MAX_WORKERS || live < 0 || live > n_shards)
     return ANTDT_ERR_INVALID_ARG;
   int64_t per = B * M;
   if (n_shards != N / per + (N % per ? 1 : 0)) return ANTDT_ERR_INVALID_ARG;
-  if (len != 8 * (10 + 2 * (size_t)n_shards + (size_t)live + 2 * (size_t)K))
+  if (len != 8 * (10 + 2 * (size_t)n_shards + (size_t)live + (3 + MAX_FINISHED) * (size_t)K))
     return ANTDT_ERR_INVALID_ARG;
   antdt_dds* d = dds_alloc(n_shards, (int32_t)K, n_shards + 16);
   if (!d) return ANTDT_ERR_INVALID_ARG;
@@ -398,6 +436,20 @@ int32_t antdt_dds_load(antdt_dds** out, const void* buf, size_t len) {
     if (u < 0 || (d->held[i] >= 0 && u >= d->shard_len[d->held[i]])) bad = 1;
     d->used[i] = u;
   }
+  for (int64_t i = 0; i < K; ++i) {
+    int64_t nf = w[k++];
+    if (nf < 0 || nf > MAX_FINISHED) { bad = 1; nf = 0; }
+    d->n_fin[i] = (int32_t)nf;
+  }
+  for (int64_t i = 0; i < K; ++i)
+    for (int32_t f = 0; f < MAX_FINISHED; ++f) {
+      int64_t j = w[k++];
+      if (f < d->n_fin[i] && (j < 0 || j >= n_shards || d->shard_state[j] != ANTDT_SHARD_DONE)) {
+        bad = 1;
+        j = 0;
+      }
+      d->fin[(size_t)i * MAX_FINISHED + f] = j;
+    }
   if (bad) { dds_free(d); return ANTDT_ERR_INVALID_ARG; }
   *out = d;
   return ANTDT_OK;

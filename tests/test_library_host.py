@@ -122,10 +122,13 @@ def test_shard_plans_match_checker_through_a_whole_epoch_with_requeues(seed):
         if rc_a == 7:
             break
         assert sum(bs_b) == B_
-        for s, n in rg_b:
-            cover[s:s + n] += 1
-        if rng.random() < 0.15:
-            w = int(rng.integers(0, K))
+        # a dropped worker's samples of this step are in no gradient that arrived
+        w = int(rng.integers(0, K)) if rng.random() < 0.15 else -1
+        for i in range(K):
+            if i != w:
+                for s, n in rg_b[ro_b[i]:ro_b[i + 1]]:
+                    cover[s:s + n] += 1
+        if w >= 0:
             a.requeue_worker(w)
             b.antdt_dds_requeue_worker(w)
             for j in range(a.num_shards()):
@@ -173,6 +176,16 @@ def test_save_load_round_trip_mid_epoch():
         assert ra == rb
         if ra[0] == B.ERR_EXHAUSTED:
             break
+    # the image carries the shards each worker finished in the latest plan call: a drop reported
+    # after a restore takes them back exactly as it would have before the save
+    d = B.Dds(600, 100, 1, 2)
+    d.antdt_shard_plan([3.0, 1.0])
+    d.antdt_shard_plan([3.0, 1.0])                 # worker 0 finishes shard 0 here
+    e = B.Dds.antdt_dds_load(d.antdt_dds_save(), 2)
+    d.antdt_dds_requeue_worker(0)
+    e.antdt_dds_requeue_worker(0)
+    assert d.antdt_dds_shard_info(0)[:2] == (B.SHARD_TODO, -1)
+    assert e.antdt_dds_save() == d.antdt_dds_save()
     with pytest.raises(B.AntdtError):
         B.Dds.antdt_dds_load(img[:-8], 6)
     with pytest.raises(B.AntdtError):

@@ -125,15 +125,18 @@ def _run_epoch(d, K, N, rng, speeds_fn, requeue_prob=0.0, rule="proportional"):
             break
         assert rc == 0
         assert bsz.sum() == d_B(d)
+        # a dropped worker's gradient never arrives: its samples of this step do not count
+        dropped = int(rng.integers(0, K)) if requeue_prob and rng.random() < requeue_prob else -1
         for i in range(K):
             got = 0
             for s, n in rg[ro[i]:ro[i + 1]]:
-                cover[s:s + n] += 1
+                if i != dropped:
+                    cover[s:s + n] += 1
                 got += n
             assert got == cnt[i] <= bsz[i]
         steps += 1
-        if requeue_prob and rng.random() < requeue_prob:
-            d.requeue_worker(int(rng.integers(0, K)))
+        if dropped >= 0:
+            d.requeue_worker(dropped)
         assert steps < 100000
     return cover, steps
 
@@ -166,6 +169,43 @@ def test_at_least_once_with_requeues_and_done_count():
     cover, _ = _run_epoch(d, K, N, rng, lambda: np.exp(rng.normal(0, 0.7, size=K)), 0.3)
     assert np.all(cover >= 1) and cover.max() >= 2
     assert d.counts() == (0, 0, -(-N // (B * M)))
+
+
+def test_drop_on_the_step_that_finishes_a_shard_loses_no_sample():
+    # 6 shards of 100 samples (M = 1), speeds 3:1 -> batches 75 / 25.  Step 1: worker 0 takes
+    # 0..74 of shard 0.  Step 2: it takes 75..99 (shard 0 finished) and 200..249 of shard 2; its
+    # gradient is then dropped.  Samples 75..99 were in no gradient that arrived, so shard 0 must
+    # come back although its last sample was served (Section V-C.3: DONE needs the push).
+    N, B, M, K = 600, 100, 1, 2
+    d = _mk(N, B, M, K)
+    cover = np.zeros(N, np.int64)
+    step = 0
+    while True:
+        rc, bsz, ro, rg, cnt = d.plan([3.0, 1.0])
+        if rc == 7:
+            break
+        step += 1
+        drop = 0 if step == 2 else -1
+        if step == 2:
+            assert rg[ro[0]:ro[1]].tolist() == [[75, 25], [200, 50]]
+            assert d.shard_info(0)[0] == 2                       # provisionally DONE
+        for i in range(K):
+            for s, n in rg[ro[i]:ro[i + 1]]:
+                if i != drop:
+                    cover[s:s + n] += 1
+        if drop >= 0:
+            d.requeue_worker(drop)
+            # both come back, the finished one first, behind the shards still queued
+            assert d.shard_info(0)[:2] == (0, -1) and d.shard_info(2)[:2] == (0, -1)
+    assert np.all(cover >= 1)
+    assert cover[:75].tolist() == [2] * 75 and cover[75:100].tolist() == [1] * 25
+    assert d.counts() == (0, 0, 6)
+    # a requeue that comes after the NEXT plan call no longer touches what that worker finished
+    d = _mk(N, B, M, K)
+    d.plan([3.0, 1.0]); d.plan([3.0, 1.0]); d.plan([3.0, 1.0])
+    assert d.shard_info(0)[0] == 2
+    d.requeue_worker(0)
+    assert d.shard_info(0)[0] == 2
 
 
 def test_doing_shard_is_exclusive_and_requeue_goes_to_queue_end():
