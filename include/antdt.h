@@ -59,7 +59,8 @@ enum {
   ANTDT_ERR_TIMEOUT = 6,             /* a bounded device-side wait ran out                */
   ANTDT_ERR_EXHAUSTED = 7,           /* the shard queue is empty: the epoch is over       */
   ANTDT_ERR_STATE = 8,               /* call not valid in the handle's current state      */
-  ANTDT_ERR_BAD_OFFSETS = 9,         /* device saw bag offsets that do not ascend / fit   */
+  ANTDT_ERR_BAD_OFFSETS = 9,         /* device saw bag offsets (or sorted id lists) that
+                                        do not ascend / fit                               */
   ANTDT_ERR_INFEASIBLE = 10          /* a planning problem has no feasible point          */
 };
 
@@ -273,7 +274,10 @@ int32_t antdt_embbag_bwd_dedup_static(const int32_t* row_ids, int64_t nnz,
  *     G = sum_i (b_i / sum_j b_j) * G_i.
  * Sparse part: agg_ids = ascending union of the workers' row lists, a worker that does not
  * hold a row contributes nothing; summed in ascending worker order.  Dense part: the same
- * weights over K dense vectors.  Either part may be NULL.
+ * weights over K dense vectors.  Either part may be NULL.  Every worker's list must ascend
+ * strictly (what antdt_embbag_bwd_dedup writes does); a list of up to 32 workers that repeats
+ * ids so often that a stretch of 4096 consecutive row ids holds more entries than K times
+ * its width raises BAD_OFFSETS in dev_status and that stretch is left out of the result.
  *   batch_sizes host [K] int64: the b_i actually served this step (counts), sum > 0. */
 typedef struct {
   int32_t dim;
@@ -387,8 +391,12 @@ int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream);
  * captures antdt_bsp_step_device on `stream` (thread-local capture mode), instantiates the graph
  * and launches it; later calls whose descriptor is equal launch the kept executable graph.
  *   - "Equal" covers every scalar and device pointer the device step reads, and the CONTENTS of
- *     worker_sample_offsets[K+1] and batch_sizes[K] (they travel as kernel parameters); `step` is
- *     compared only for Adam.  What the device pointers point at may differ from call to call.
+ *     worker_sample_offsets[K+1] and batch_sizes[K] (they travel as kernel parameters); the
+ *     value of `step` is not part of it.  What the device pointers point at may differ from
+ *     call to call.
+ *   - opt == ANTDT_OPT_ADAM is issued as the plain launches of antdt_bsp_step_device: its bias
+ *     corrections change with every step and are kernel parameters, so no graph could be
+ *     replayed and a capture per step costs more than it saves.
  *   - Up to 8 executable graphs are kept per device, least recently used replaced; a replaced
  *     one is updated in place when the new capture has the same shape, else re-instantiated.  A
  *     descriptor that changes every step therefore still runs as a graph, at the host cost of one

@@ -38,6 +38,9 @@ _lib.orc_embbag_fwd.argtypes = [_p, C.c_int, C.c_int64, C.c_int, _p, _p, C.c_int
 _lib.orc_embbag_bwd_dedup.restype = C.c_int64
 _lib.orc_embbag_bwd_dedup.argtypes = [_p, _p, C.c_int64, C.c_int, _p, C.c_int, C.c_int64, C.c_int,
                                       _p, _p, _p, _p, _p, _p, C.c_int64]
+_lib.orc_embbag_bwd_accum.restype = C.c_int64
+_lib.orc_embbag_bwd_accum.argtypes = [_p, _p, C.c_int64, C.c_int, _p, C.c_int, C.c_int64, C.c_int,
+                                      _p, _p, _p, _p, _p, C.c_int64]
 _lib.orc_aggregate_sparse.restype = C.c_int64
 _lib.orc_aggregate_sparse.argtypes = [C.c_int, _p, _p, _p, _p, C.c_int, _p, _p, C.c_int64]
 _lib.orc_aggregate_dense.argtypes = [_p, C.c_int64, C.c_int64, _p, C.c_int, _p]
@@ -160,6 +163,28 @@ def embbag_bwd_dedup(row_ids, bag_offsets, F, d_pooled, n_rows, worker_sample_of
         raise OracleError(-nu)
     return dict(uniq_ids=uid[:nu].copy(), worker_uniq_offsets=wuo, seg_offsets=so[: nu + 1].copy(),
                 sorted_occ=occ[:nnz].copy(), uniq_grads=ug[:nu].copy())
+
+
+def embbag_bwd_accum(row_ids, bag_offsets, F, d_pooled, n_rows, worker_sample_offsets, micro_batches):
+    """Gradient accumulation (Section VI-B): worker w's samples are micro_batches[w] micro-batches
+    back to back; -> dict(uniq_ids, worker_uniq_offsets, uniq_grads), the mean of the micro-batch
+    mean gradients."""
+    n_bags = bag_offsets.shape[0] - 1
+    nnz = int(bag_offsets[-1])
+    D = d_pooled.shape[1]
+    K = worker_sample_offsets.shape[0] - 1
+    cap = max(nnz, 1)
+    uid = np.zeros(cap, _i32)
+    wuo = np.zeros(K + 1, _i64)
+    ug = np.zeros((cap, D), _f32)
+    nu = _lib.orc_embbag_bwd_accum(_ptr(_chk(row_ids, _i32)), _ptr(_chk(bag_offsets, _i64)), n_bags,
+                                   F, _ptr(_chk(d_pooled, _f32)), D, n_rows, K,
+                                   _ptr(_chk(worker_sample_offsets, _i64)),
+                                   _ptr(np.ascontiguousarray(micro_batches, _i64)), _ptr(uid),
+                                   _ptr(wuo), _ptr(ug), cap)
+    if nu < 0:
+        raise OracleError(-nu)
+    return dict(uniq_ids=uid[:nu].copy(), worker_uniq_offsets=wuo, uniq_grads=ug[:nu].copy())
 
 
 def aggregate_sparse(uniq_ids, worker_uniq_offsets, uniq_grads, batch_sizes_):

@@ -21,6 +21,7 @@
 #include <cstring>
 #include <deque>
 #include <limits>
+#include <map>
 #include <utility>
 #include <vector>
 
@@ -396,6 +397,52 @@ i64 orc_embbag_bwd_dedup(const i32* ids, const i64* off, i64 n_bags, int F, cons
   }
   wuo[K] = nu;
   seg_off[nu] = off[n_bags];
+  return nu;
+}
+
+// AntDT-DD with gradient accumulation (Section VI-B, the paragraph before Eq. 4): a device whose
+// plan is (B_w, C_w) runs C_w micro-batches of B_w samples between two synchronisations and
+// pushes the accumulated gradient.  Worker w's samples [wso[w], wso[w+1]) are its C_w micro-batches
+// back to back (so C_w divides their number); each micro-batch yields its own mean gradient over
+// its B_w samples, and the pushed gradient is the mean of those C_w means.  A row that a
+// micro-batch does not touch gets zero from it.  Distinct rows ascending per worker, as above.
+// Returns the number of (worker, row) pairs, or -(error code).
+i64 orc_embbag_bwd_accum(const i32* ids, const i64* off, i64 n_bags, int F, const float* dY, int dim,
+                         i64 n_rows, int K, const i64* wso, const i64* micro, i32* uniq_ids,
+                         i64* wuo, float* uniq_grads, i64 cap) {
+  int rc = check_bags(ids, off, n_bags, n_rows);
+  if (rc != OK) return -rc;
+  if (wso[0] != 0 || wso[K] * F != n_bags) return -E_ARG;
+  i64 nu = 0;
+  for (int w = 0; w < K; ++w) {
+    wuo[w] = nu;
+    const i64 n_w = wso[w + 1] - wso[w], C = micro[w];
+    if (C < 1 || n_w % C != 0) return -E_ARG;
+    const i64 Bw = n_w / C;
+    std::map<i32, std::vector<double> > pushed;  // sum over micro-batches of their mean gradients
+    for (i64 c = 0; c < C; ++c) {
+      std::map<i32, std::vector<double> > local;  // this micro-batch's gradient SUM per row
+      const i64 s0 = wso[w] + c * Bw;
+      for (i64 b = s0 * F; b < (s0 + Bw) * F; ++b)
+        for (i64 j = off[b]; j < off[b + 1]; ++j) {
+          std::vector<double>& g = local[ids[j]];
+          if (g.empty()) g.assign(dim, 0.0);
+          for (int e = 0; e < dim; ++e) g[e] += (double)dY[b * dim + e];
+        }
+      for (const auto& kv : local) {
+        std::vector<double>& g = pushed[kv.first];
+        if (g.empty()) g.assign(dim, 0.0);
+        for (int e = 0; e < dim; ++e) g[e] += kv.second[e] / (double)Bw;  // the micro-batch mean
+      }
+    }
+    for (const auto& kv : pushed) {
+      if (nu >= cap) return -E_CAP;
+      uniq_ids[nu] = kv.first;
+      for (int e = 0; e < dim; ++e) uniq_grads[nu * dim + e] = (float)(kv.second[e] / (double)C);
+      ++nu;
+    }
+  }
+  wuo[K] = nu;
   return nu;
 }
 

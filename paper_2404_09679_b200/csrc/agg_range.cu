@@ -263,6 +263,13 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   const int64_t u0 = __ldg(base + b);  // requested now: every global round trip here is serial
   const Pieces pc = range_pieces(bnd, wuo, K, P, b, dropped, s_beg, s_off, s_before);
   if (pc.entries == 0) return;
+  // A worker lists a row id at most once, so a range holds at most R*K entries and the arrays
+  // below are sized for that.  More means a list that does not strictly ascend: flag it and
+  // leave the range out (its slots keep the zeroed head bits; the reduction bounds every index).
+  if (pc.entries > (K << r_log2)) {
+    if (tid == 0) set_status(status, ANTDT_ERR_BAD_OFFSETS);
+    return;
+  }
   // hb word i is global head-bit word (before >> 5) + i, same bit positions
   const int hb_shift = (int)(pc.before & 31);
   const int n_hw = (hb_shift + pc.entries + 31) >> 5;

@@ -131,6 +131,7 @@ int32_t bwd_dedup_impl(
   if (!bag_offsets || !worker_sample_offsets || !worker_uniq_offsets || !seg_offsets || !ws)
     return ANTDT_ERR_INVALID_ARG;
   if (nnz > 0 && (!row_ids || !d_pooled || !sorted_occ)) return ANTDT_ERR_INVALID_ARG;
+  if (nnz > 0 && n_bags == 0) return ANTDT_ERR_INVALID_ARG;  // occurrences that belong to no bag
   if (out_cap > 0 && (!uniq_ids || !uniq_grads)) return ANTDT_ERR_INVALID_ARG;
   if (!aligned16(d_pooled) || !aligned16(uniq_grads) || !aligned16(ws)) return ANTDT_ERR_INVALID_ARG;
   if (worker_sample_offsets[0] != 0) return ANTDT_ERR_INVALID_ARG;

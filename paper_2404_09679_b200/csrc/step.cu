@@ -218,12 +218,11 @@ std::vector<uint64_t> graph_key(const antdt_step_desc* d) {
   std::vector<uint64_t> k;
   const int K = d->n_workers;
   k.reserve(48 + 2 * (size_t)K);
-  const bool adam = d->opt == ANTDT_OPT_ADAM;
   const uint64_t head[] = {
       bits_of(d->table), (uint64_t)d->dtype, (uint64_t)d->n_rows, (uint64_t)d->dim,
       bits_of(d->state0), bits_of(d->state1), (uint64_t)d->opt, bits_of(d->lr), bits_of(d->eps),
       bits_of(d->beta1), bits_of(d->beta2),
-      adam ? (uint64_t)d->step : (uint64_t)(d->step >= 1),  // Adagrad does not use the step number
+      (uint64_t)(d->step >= 1),  // the Adagrad variants do not use the step number
       (uint64_t)d->nnz, (uint64_t)d->n_bags, (uint64_t)d->bags_per_sample, (uint64_t)d->dense_n,
       (uint64_t)K, bits_of(d->d_row_ids), bits_of(d->d_bag_offsets), bits_of(d->d_pooled_out),
       bits_of(d->d_d_pooled), bits_of(d->d_dense_grads), bits_of(d->d_dense_out),
@@ -250,6 +249,9 @@ extern "C" int32_t antdt_bsp_step_graph(const antdt_step_desc* d, void* stream) 
   }
   // inside somebody else's capture the launches simply join that graph
   if (cs != cudaStreamCaptureStatusNone) return antdt_bsp_step_device(d, stream);
+  // Adam's bias corrections depend on the step number and travel as kernel parameters, so no two
+  // steps share a graph: a capture per step would cost more than the launches it replaces
+  if (d->opt == ANTDT_OPT_ADAM) return antdt_bsp_step_device(d, stream);
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ANTDT_ERR_CUDA;
   const std::vector<uint64_t> key = graph_key(d);

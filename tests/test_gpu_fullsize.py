@@ -158,7 +158,8 @@ def test_full_size_step(cfg):
         G.close_mostly(a, b, G.BF16_RTOL, 1e-6, 1e-3, 2 * w.lr)
     else:
         G.close_mostly(got, tR, 5e-5, 2e-6, 1e-3, 2 * w.lr)
-    G.close_mostly(s0[R].cpu().numpy(), r0, 1e-4, 1e-7, 1e-3, 1.0)
+    # the state is well conditioned: no element may leave a band of the tolerance's own size
+    G.close_mostly(s0[R].cpu().numpy(), r0, 1e-4, 1e-7, 1e-3, 1e-6 + 1e-4 * float(np.abs(r0).max()))
     # rows outside the batch: bit-identical
     assert torch.equal(table[untouched_probe].view(torch.int16 if w.table_dtype == "bf16" else torch.int32),
                        t_before_probe.view(torch.int16 if w.table_dtype == "bf16" else torch.int32))

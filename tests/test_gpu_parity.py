@@ -193,6 +193,11 @@ def test_bwd_flags_bad_ids_and_capacity():
     off_bad = off.copy()
     off_bad[5] = off_bad[6] + 1
     assert G.gpu_bwd(ids, off_bad, F, dY, V, wso)["status"] == B.ERR_BAD_OFFSETS
+    # occurrences without a single bag to belong to: refused on the host, nothing is launched
+    with pytest.raises(B.AntdtError) as ei:
+        G.gpu_bwd(ids[:5], np.zeros(1, np.int64), F, np.zeros((1, D), np.float32), V,
+                  np.array([0, 0], np.int64))
+    assert ei.value.code == B.ERR_INVALID_ARG
 
 
 # ---- aggregation ---------------------------------------------------------------------------
@@ -282,6 +287,18 @@ def test_sparse_aggregate_flags_ids_outside_the_table():
     want_ids, want = oracle.aggregate_sparse(uid, wuo, g, [1] * K)
     assert code == 0 and np.array_equal(ids, want_ids)
     G.close(agg, want)
+
+
+def test_sparse_aggregate_flags_a_list_that_repeats_ids():
+    """A worker list must ascend strictly.  One that repeats an id 9000 times puts more entries
+    into a 4096-id stretch than 2 workers can legitimately list there: flagged (only the status
+    word is specified), every access stays inside the buffers."""
+    D = 4
+    uid = np.concatenate([np.full(9000, 7, np.int32), np.array([3, 9], np.int32)])
+    wuo = np.array([0, 9000, 9002], np.int64)
+    g = np.ones((len(uid), D), np.float32)
+    _, _, _, _, code = G.gpu_aggregate(uid, wuo, g, [1, 1], 50_000)
+    assert code == B.ERR_BAD_OFFSETS
 
 
 def test_aggregate_invariants_on_gpu():

@@ -102,7 +102,11 @@ def test_steps_match_checker(name):
             G.close_mostly(a, b, G.BF16_RTOL, 1e-6, 1e-3, 2 * w.lr)
         else:
             G.close_mostly(got_rows, ref.table[want["agg_ids"]], 5e-5, 2e-6, 1e-3, 2 * w.lr)
-        G.close_mostly(s0[rows].cpu().numpy(), ref.s0[want["agg_ids"]], 1e-4, 1e-7, 1e-3, 1.0)
+        # the state is well conditioned (acc += g^2 and m += (1-b1) g move by at most 2|g| dg + dg^2
+        # and dg for a gradient off by dg): no element may leave a band of the tolerance's own size
+        s0_want = ref.s0[want["agg_ids"]]
+        G.close_mostly(s0[rows].cpu().numpy(), s0_want, 1e-4, 1e-7, 1e-3,
+                       1e-6 + 1e-4 * float(np.abs(s0_want).max()))
         # --- (2) free-running trajectory -----------------------------------------------------
         run_step(buf, free_t, free_s0, free_s1, oc, s + 1, batch["row_ids"], batch["bag_offsets"],
                  w.F, batch["d_pooled"], batch["wso"].tolist(), batch["counts"].tolist(),

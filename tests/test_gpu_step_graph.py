@@ -5,8 +5,9 @@ The kernels are deterministic, so the two launch forms must agree bit for bit on
 and on the table and optimizer state after every step.  The cases cover the three ways a call
 meets the graph store: a descriptor seen before (replay), a new descriptor while slots are free
 (instantiate), and a new descriptor once the 8 slots are taken (least recently used graph
-updated in place) - including batches whose sizes differ from step to step and Adam, whose
-step number changes the kernel parameters every step."""
+updated in place) - including batches whose sizes differ from step to step - and Adam, which
+the entry point issues as plain launches (its step number changes kernel parameters every
+step, so no graph could be replayed)."""
 import numpy as np
 import pytest
 import torch
@@ -24,7 +25,7 @@ CASES = {
     "c1_varying_sizes": (synth.WORKLOADS[1], 12, 12),
     # fixed sizes, two batches in rotation: every step after the first two is a replay
     "c2_replay": (synth.WORKLOADS[2].scaled(V=26 * 50_000), 8, 2),
-    # Adam + dense part: the step number changes the captured parameters every step
+    # Adam + dense part: issued as plain launches by the entry point
     "c3_adam_dense": (synth.WORKLOADS[3].scaled(B=2048, V=200_000, dense_n=65_536), 10, 3),
 }
 

@@ -123,6 +123,44 @@ def test_bwd_all_ids_distinct_is_a_scaled_copy():
         assert np.array_equal(r["uniq_grads"][lo:hi], want)
 
 
+# ---- gradient accumulation (AntDT-DD, Section VI-B) ------------------------------------------
+def test_accumulated_gradient_is_the_mean_over_all_micro_batch_samples():
+    # C_w micro-batches of B_w samples each: the mean of the C_w means is the mean over the
+    # C_w * B_w samples, which the dense count matrix gives without any notion of micro-batches
+    rng = np.random.default_rng(30)
+    V, D, F = 30, 4, 3
+    micro = np.array([3, 1, 2, 4], np.int64)
+    bsz = np.array([4, 7, 5, 2], np.int64)                 # B_w
+    wso = np.concatenate([[0], np.cumsum(micro * bsz)]).astype(np.int64)
+    S = int(wso[-1])
+    ids, off = random_bags(rng, S * F, V, 4, zipf=1.3)
+    dY = rng.normal(size=(S * F, D)).astype(np.float32)
+    r = oracle.embbag_bwd_accum(ids, off, F, dY, V, wso, micro)
+    uniq, grads, _, wuo, _ = _brute_bwd(ids, off, F, dY, V, wso)
+    assert np.array_equal(r["uniq_ids"], uniq) and np.array_equal(r["worker_uniq_offsets"], wuo)
+    assert np.allclose(r["uniq_grads"], grads, rtol=1e-6, atol=1e-9)
+    # without accumulation it IS the plain backward, value for value
+    one = oracle.embbag_bwd_accum(ids, off, F, dY, V, wso, np.ones(4, np.int64))
+    plain = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+    assert np.array_equal(one["uniq_ids"], plain["uniq_ids"])
+    assert np.array_equal(one["uniq_grads"], plain["uniq_grads"])
+    # a micro-batch count that does not divide the worker's samples is refused
+    with pytest.raises(oracle.OracleError):
+        oracle.embbag_bwd_accum(ids, off, F, dY, V, wso, np.array([5, 1, 2, 4], np.int64))
+
+
+def test_accumulation_hand_case_with_a_row_missing_from_a_micro_batch():
+    # one worker, 2 micro-batches of 2 samples, one bag per sample, dim 1.
+    # row 5 occurs in samples 0, 1 and 3 (dY 1, 2, 8), row 9 only in sample 2 (dY 4):
+    #   micro-batch means: row 5 -> (1+2)/2 = 1.5 and 8/2 = 4 ; row 9 -> 0 and 4/2 = 2
+    #   pushed = mean of the two: row 5 -> 2.75, row 9 -> 1.0
+    ids = np.array([5, 5, 9, 5], np.int32)
+    off = np.arange(5, dtype=np.int64)
+    dY = np.array([[1.0], [2.0], [4.0], [8.0]], np.float32)
+    r = oracle.embbag_bwd_accum(ids, off, 1, dY, 10, np.array([0, 4], np.int64), np.array([2], np.int64))
+    assert r["uniq_ids"].tolist() == [5, 9] and r["uniq_grads"][:, 0].tolist() == [2.75, 1.0]
+
+
 # ---- aggregation ---------------------------------------------------------------------------
 def test_weighted_aggregate_equals_full_batch_mean_gradient():
     rng = np.random.default_rng(30)

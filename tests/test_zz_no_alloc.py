@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2404_09679_b200 import binding as B
 from tests import gpu_util as G
 from tests.util import random_bags
@@ -47,13 +48,22 @@ def _problem(seed, V, D, K, F, S, maxlen, zipf):
 
 def test_static_scratch_variant_matches_the_workspace_variant_twice_in_a_row():
     # first a large problem (long runs, many tiles), then a smaller, differently shaped one
-    for args in (_problem(1, 3000, 64, 8, 6, 20_000, 9, 1.15), _problem(2, 50_000, 16, 3, 4, 5000, 5, None)):
+    for n, args in enumerate((_problem(1, 3000, 64, 8, 6, 20_000, 9, 1.15),
+                              _problem(2, 50_000, 16, 3, 4, 5000, 5, None))):
         want = G.gpu_bwd(*args)
         assert want["status"] == 0
         got = _static_bwd(*args)
         for k in ("worker_uniq_offsets", "uniq_ids", "seg_offsets", "sorted_occ"):
             assert np.array_equal(got[k], want[k]), k
         G.close(got["uniq_grads"], want["uniq_grads"])
+        if n == 1:
+            # the call that found leftovers in the scratch, against the CPU checker as well, so
+            # that this file stands on its own
+            ids, off, F, dY, V, wso = args
+            ref = oracle.embbag_bwd_dedup(ids, off, F, dY, V, wso)
+            for k in ("worker_uniq_offsets", "uniq_ids", "seg_offsets", "sorted_occ"):
+                assert np.array_equal(got[k], ref[k]), k
+            G.close(got["uniq_grads"], ref["uniq_grads"])
 
 
 def test_static_scratch_variant_rejects_what_does_not_fit():
