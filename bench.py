@@ -153,10 +153,93 @@ def plan_all(w, n_steps):
     return plans
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
-# full-size default workload summarised in profiles/; a kernel that has changed since is set to None.
-NCU_TRAFFIC = {4: {"seg_reduce_tiles": 12.80e9, "agg_reduce": 6.77e9, "sparse_adagrad": 9.41e9,
-                   "embbag_fwd": 4.04e9, "radix_scatter": 2.44e9}}
+def plan_all_checker(w, n_steps):
+    """The same plans from the CPU checker's own planner: the reference arm never loads the
+    CUDA library."""
+    import oracle
+    from paper_2404_09679_b200 import synth
+    dds = oracle.Dds(w.n_samples, w.B, w.M, w.K, 0)
+    plans = []
+    for s in range(n_steps):
+        v = synth.speeds_for_step(w, s)
+        rc, bsz, ro, rg, cnt = dds.plan(v, w.rule, w.min_batch, cap=4 * w.K + 16)
+        assert rc == 0 and int(bsz.sum()) == w.B
+        plans.append(dict(speeds=v, batch_sizes=[int(x) for x in bsz], counts=[int(x) for x in cnt],
+                          ranges=[(int(a), int(b)) for a, b in rg]))
+    return plans
+
+
+def host_info():
+    """CPU model and core counts of the box the checker is timed on."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for ln in f:
+                if ln.lower().startswith("model name"):
+                    model = ln.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    try:
+        usable = len(os.sched_getaffinity(0))
+    except (AttributeError, OSError):
+        usable = os.cpu_count() or 1
+    return {"cpu_model": model, "cores_total": os.cpu_count() or 1, "cores_usable": usable}
+
+
+class PinnedToOneCore:
+    """Pins this process to one of its allowed cores for the checker's timed leg (the checker is
+    single-threaded; pinning keeps the scheduler from migrating it) and restores the mask."""
+
+    def __enter__(self):
+        self.old, self.core = None, None
+        try:
+            self.old = os.sched_getaffinity(0)
+            self.core = sorted(self.old)[-1]
+            os.sched_setaffinity(0, {self.core})
+        except (AttributeError, OSError):
+            self.old = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.old is not None:
+            try:
+                os.sched_setaffinity(0, self.old)
+            except OSError:
+                pass
+        return False
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) come from ncu captures
+# summarised in profiles/dram_traffic.json, which records for every kernel the hash of the source
+# files it was compiled from: a kernel whose sources have changed since reports no traffic.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+CSRC = os.path.join(ROOT, "paper_2404_09679_b200", "csrc")
+
+
+def sources_hash(files):
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(files):
+        try:
+            with open(os.path.join(CSRC, f), "rb") as g:
+                h.update(g.read())
+        except OSError:
+            h.update(b"missing:" + f.encode())
+    return h.hexdigest()[:16]
+
+
+def load_traffic(cfg):
+    """-> {kernel: bytes per launch} for this config, only kernels whose sources are unchanged."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        return {}, None
+    out = {}
+    for name, k in rec.get("configs", {}).get(str(cfg), {}).items():
+        if sources_hash(k.get("sources", [])) == k.get("sources_sha"):
+            out[name] = float(k["dram_bytes_per_launch"])
+    return out, rec.get("commit")
 
 
 def scaled_workload(w, scale):
@@ -279,9 +362,11 @@ REF_SAMPLE_PER_WORKER = {1: 1 << 30, 2: 1 << 30, 3: 256, 4: 256, 5: 1536}
 def cpu_baseline(w, cfg, bm, plan, table):
     repeats = 5 if cfg <= 2 else 1
     smp = OracleSample(w, bm, plan, table, CPU_SAMPLE_PER_WORKER[cfg])
-    ts = [smp.run(s + 1) for s in range(repeats)]
+    with PinnedToOneCore() as pin:
+        ts = [smp.run(s + 1) for s in range(repeats)]
     t = statistics.median(ts)
     return {"value": smp.n_samples / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "pinned_to_core": pin.core, **host_info(),
             "sample": f"first {min(CPU_SAMPLE_PER_WORKER[cfg], max(plan['counts']))} samples of each "
                       f"of the {w.K} workers of one batch ({smp.n_samples} samples, "
                       f"{len(smp.ids)} occurrences, touched rows only"
@@ -443,34 +528,71 @@ def run_ours(args):
     nnz_avg = sum(b["ids"].numel() for b in batches) / n_batches
     bags_avg = sum(b["off"].numel() - 1 for b in batches) / n_batches
     alg = algorithmic_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen)
+    traffic, traffic_commit = load_traffic(cfg) if (args.scale == 1.0 and world == 1) else ({}, None)
+    D, ew = w.D, (2 if w.table_dtype == "bf16" else 4)
+    # the two gathering kernels: bytes their gathers pull (at full multiplicity) and what a perfect
+    # cache would leave for DRAM (every distinct input row once + ids + outputs)
+    gathers = {"embbag_fwd": (nnz_avg * D * ew, D * ew,
+                              4 * nnz_avg + 8 * (bags_avg + 1) + u_seen * D * ew + bags_avg * D * 4),
+               "seg_reduce_tiles": (nnz_avg * D * 4, D * 4,
+                                    4 * nnz_avg + nnz_avg / 8 + bags_avg * D * 4 + sum_u_seen * D * 4)}
     kern = {}
+    step_dram, step_dram_missing = 0.0, []
     for name, (n, tms) in prof.items():
         d = {"launches": n, "ms_total": round(tms, 4), "share": round(tms / max(prof_ms, 1e-9), 4)}
         if name in alg and n:
             d["algorithmic_GBps"] = round(alg[name] / (tms / n * 1e-3) / 1e9, 1)
+        if name in traffic and n:
+            d["dram_GBps"] = round(traffic[name] / (tms / n * 1e-3) / 1e9, 1)
+            d["dram_frac"] = round(d["dram_GBps"] / peak_gbs, 4)
+            step_dram += traffic[name] * n / K_steps
+        elif tms / max(prof_ms, 1e-9) > 0.005:
+            step_dram_missing.append(name)
         kern[name] = d
     top = max(prof.items(), key=lambda kv: kv[1][1])[0]
     top_n, top_ms = prof[top]
+    top_s = top_ms / top_n * 1e-3
     roof = {"kernel": top, "bound": "hbm", "unit": "GB/s", "peak": peak_gbs,
             "peak_source": "MEASURED_PEAKS.json hbm_gbs (measured copy)" if peaks else "fallback 6650",
-            "achieved": None, "frac": None, "traffic": None,
+            "achieved": None, "frac": None, "traffic": traffic.get(top),
             "algorithmic_bytes_per_launch": alg.get(top), "avg_launch_ms": round(top_ms / top_n, 4)}
     if top in alg:
-        roof["achieved"] = round(alg[top] / (top_ms / top_n * 1e-3) / 1e9, 1)
+        roof["achieved_algorithmic"] = round(alg[top] / top_s / 1e9, 1)
+        roof["frac_algorithmic"] = round(roof["achieved_algorithmic"] / peak_gbs, 4)
+    if top in gathers:
+        roof["compulsory_bytes_per_launch"] = int(gathers[top][2])
+        roof["frac_compulsory"] = round(gathers[top][2] / top_s / 1e9 / peak_gbs, 4)
+    # `frac` is what DRAM did: measured DRAM bytes where a capture of this kernel exists; else, for
+    # a gathering kernel (whose repeats are served by L1/L2, so its algorithmic rate is not a DRAM
+    # rate), the compulsory bytes; else the algorithmic bytes (streaming kernels: the same thing)
+    if roof["traffic"]:
+        roof["achieved"] = round(roof["traffic"] / top_s / 1e9, 1)
+        roof["frac_source"] = (f"ncu dram bytes per launch (profiles/dram_traffic.json, commit "
+                               f"{traffic_commit}) / CUDA-event launch time")
+    elif top in gathers:
+        roof["achieved"] = round(gathers[top][2] / top_s / 1e9, 1)
+        roof["frac_source"] = ("compulsory bytes (every distinct input row once, ids, outputs): a lower "
+                               "bound of the DRAM traffic; no current ncu capture of this kernel here")
+    elif top in alg:
+        roof["achieved"] = roof["achieved_algorithmic"]
+        roof["frac_source"] = "algorithmic bytes (a streaming kernel: every byte is touched once)"
+    if roof["achieved"] is not None:
         roof["frac"] = round(roof["achieved"] / peak_gbs, 4)
-    if top in ("seg_reduce_tiles", "embbag_fwd"):
-        roof["note"] = ("gather counted at full multiplicity; repeats of a row are served by L2, so the "
-                        "algorithmic rate can exceed the DRAM peak: see traffic and the compulsory figures")
-        # every distinct input row once + ids + outputs: what a perfect cache would leave for DRAM
-        D, ew = w.D, (2 if w.table_dtype == "bf16" else 4)
-        comp = (4 * nnz_avg + nnz_avg / 8 + bags_avg * D * 4 + sum_u_seen * D * 4 if top == "seg_reduce_tiles"
-                else 4 * nnz_avg + 8 * (bags_avg + 1) + u_seen * D * ew + bags_avg * D * 4)
-        roof["compulsory_bytes_per_launch"] = int(comp)
-        roof["frac_compulsory"] = round(comp / (top_ms / top_n * 1e-3) / 1e9 / peak_gbs, 4)
-    if args.scale == 1.0 and world == 1:
-        roof["traffic"] = NCU_TRAFFIC.get(cfg, {}).get(top)
-        if roof["traffic"]:
-            roof["dram_GBps_from_traffic"] = round(roof["traffic"] / (top_ms / top_n * 1e-3) / 1e9, 1)
+    # secondary roof of the gathering kernels: the rate at which the SMs pull scattered rows of the
+    # same width out of an L2-resident matrix (measured here with the library's plain probe)
+    l2 = None
+    if not args.no_l2_probe:
+        l2 = {}
+        for name, (gbytes, row_bytes, _) in gathers.items():
+            if name not in prof or not prof[name][0]:
+                continue
+            rate = measure_l2_gather(B, dev, row_bytes, stream)
+            n, tms = prof[name]
+            ach = gbytes / (tms / n * 1e-3) / 1e9
+            l2[name] = {"row_bytes": row_bytes, "l2_gather_peak_GBps": round(rate, 1),
+                        "gathered_GBps": round(ach, 1), "frac_of_l2_gather_peak": round(ach / rate, 4)}
+            kern[name]["frac_of_l2_gather_peak"] = l2[name]["frac_of_l2_gather_peak"]
+        roof["l2_gather"] = l2.get(top)
     rowbits = max(1, (w.V - 1).bit_length())
     passes = -(-rowbits // 9)
     sb = step_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen, passes, passes)
@@ -497,6 +619,11 @@ def run_ours(args):
         "roofline": roof,
         "step_algorithmic_GB": round(sb / 1e9, 3),
         "step_GBps_algorithmic": round(sb / (ms / K_steps * 1e-3) / 1e9, 1),
+        "step_dram_GB": round(step_dram / 1e9, 3) if traffic else None,
+        "step_frac_dram": (round(step_dram / (ms / K_steps * 1e-3) / 1e9 / peak_gbs, 4)
+                           if traffic else None),
+        "step_dram_kernels_without_capture": step_dram_missing if traffic else None,
+        "l2_gather": l2,
         "kernels": kern,
         "kernels_timed_in": ("the timed steps (event pair around every launch)" if not use_graph else
                              f"the same {K_steps} steps issued again as plain launches, "
@@ -504,6 +631,35 @@ def run_ours(args):
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
+
+
+def measure_l2_gather(B, dev, row_bytes, stream, _cache={}):
+    """GB/s at which antdt_probe_gather pulls uniformly random rows of `row_bytes` out of a 32 MB
+    matrix (L2 resident after the first touch); best of 5 launches of about 4 GB each."""
+    if row_bytes in _cache:
+        return _cache[row_bytes]
+    dim = row_bytes // 4
+    if dim not in (16, 32, 64, 128):
+        dim = 64
+    n_rows = (32 << 20) // (dim * 4)
+    per_out, n_out = 32, (1 << 24) // 32 * (64 // min(dim, 64))
+    g = torch.Generator(device=dev)
+    g.manual_seed(12345)
+    rows = torch.randn(n_rows, dim, device=dev, generator=g)
+    idx = torch.randint(0, n_rows, (n_out * per_out,), device=dev, generator=g, dtype=torch.int32)
+    out = torch.empty(n_out, dim, device=dev)
+    best = float("inf")
+    for i in range(8):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        B.antdt_probe_gather(rows, idx, per_out, out, stream=stream)
+        e1.record(stream)
+        e1.synchronize()
+        if i >= 3:
+            best = min(best, e0.elapsed_time(e1))
+    _cache[row_bytes] = n_out * per_out * dim * 4 / (best * 1e-3) / 1e9
+    del rows, idx, out
+    return _cache[row_bytes]
 
 
 def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream):
@@ -590,7 +746,7 @@ def run_reference(args):
     cfg = args.config
     w = scaled_workload(synth.WORKLOADS[cfg], args.scale)
     dev = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
-    plans = plan_all(w, 1)
+    plans = plan_all_checker(w, 1)
     bm = synth.BatchMaker(w, dev)
 
     class _LazyTable:                     # rows of the initial table, produced on demand
@@ -603,12 +759,13 @@ def run_reference(args):
             return (w.init_std * synth.normal01(h)).to(torch.float32).to(self.dtype)
 
     smp = OracleSample(w, bm, plans[0], _LazyTable(), REF_SAMPLE_PER_WORKER[cfg])
-    for s in range(args.warmup):
-        smp.run(s + 1)
-    t0 = time.perf_counter()
-    for s in range(args.steps):
-        smp.run(args.warmup + s + 1)
-    dt = time.perf_counter() - t0
+    with PinnedToOneCore() as pin:
+        for s in range(args.warmup):
+            smp.run(s + 1)
+        t0 = time.perf_counter()
+        for s in range(args.steps):
+            smp.run(args.warmup + s + 1)
+        dt = time.perf_counter() - t0
     value = smp.n_samples * args.steps / dt
     sample = (f"each step = first {min(REF_SAMPLE_PER_WORKER[cfg], max(plans[0]['counts']))} samples of "
               f"each of the {w.K} workers of one batch ({smp.n_samples} samples, {len(smp.ids)} "
@@ -620,7 +777,8 @@ def run_reference(args):
         "data": "synthetic",
         "config": {"workload": f"configs[{cfg - 1}] {w.name}: K={w.K} workers, B={w.B}, F={w.F}, "
                                f"V={w.V} x D={w.D} {w.table_dtype}, {w.opt}", "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "pinned_to_core": pin.core, **host_info()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -639,6 +797,8 @@ def main():
                          "for the launch-bound configs 1 and 2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-l2-probe", action="store_true",
+                    help="skip the L2 gather-rate probe (profiling runs)")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink batch, table rows and dense vector by this factor (profiling "
                          "captures on a small case); the JSON line says so")

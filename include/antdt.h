@@ -429,6 +429,15 @@ int32_t antdt_profile_enable(int32_t on);
 int32_t antdt_profile_kernels(void);
 int32_t antdt_profile_get(int32_t idx, char* name, size_t name_cap, int64_t* launches,
                           double* total_ms);
+/* Measurement aid (the paper has no counterpart): the plainest gather there is, for finding the
+ * rate at which this GPU's SMs can pull scattered rows out of L2, the ceiling that the
+ * gathering kernels of the step meet once the rows they repeat are cache resident.  Output
+ * row o = sum of the per_out rows rows[idx[o*per_out + j]] (an index outside [0, n_rows) reads
+ * row 0).  rows device [n_rows, dim] fp32, dim one of 16 / 32 / 64 / 128, 16-byte aligned;
+ * idx device [n_out*per_out] int32; out device [n_out, dim].  Time it with events on `stream`
+ * on a matrix of a few tens of MB with uniformly random idx. */
+int32_t antdt_probe_gather(const float* rows, int64_t n_rows, int32_t dim, const int32_t* idx,
+                           int64_t n_out, int32_t per_out, float* out, void* stream);
 const char* antdt_version(void);
 
 #ifdef __cplusplus

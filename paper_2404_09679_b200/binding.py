@@ -36,7 +36,8 @@ EXPORTS = [
     "antdt_weighted_aggregate_backup",
     "antdt_sparse_opt_update", "antdt_dense_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_bsp_step_graph", "antdt_bsp_step_graph_reset",
     "antdt_read_status", "antdt_launch_count",
-    "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_version",
+    "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_probe_gather",
+    "antdt_version",
 ]
 
 
@@ -145,6 +146,8 @@ def lib() -> C.CDLL:
         L.antdt_profile_enable.argtypes = [I32]
         L.antdt_profile_get.argtypes = [I32, C.c_char_p, SZ, C.POINTER(I64), C.POINTER(D)]
         L.antdt_version.restype = C.c_char_p
+        L.antdt_probe_gather.argtypes = [P, I64, I32, P, I64, I32, P, P]
+        L.antdt_probe_gather.restype = I32
         for fn in ("antdt_ctl_create", "antdt_ctl_report", "antdt_ctl_decide",
                    "antdt_dds_create", "antdt_batch_sizes", "antdt_shard_plan",
                    "antdt_dds_requeue_worker", "antdt_dds_counts", "antdt_dds_shard_info",
@@ -446,6 +449,12 @@ def antdt_profile_get():
                "antdt_profile_get")
         out[name.value.decode()] = (launches.value, ms.value)
     return out
+
+
+def antdt_probe_gather(rows, idx, per_out: int, out, stream=None):
+    """out[o] = sum of rows[idx[o*per_out : (o+1)*per_out]]: the gather-rate probe."""
+    _check(lib().antdt_probe_gather(_dp(rows), rows.shape[0], rows.shape[1], _dp(idx), out.shape[0],
+                                    per_out, _dp(out), _stream(stream)), "antdt_probe_gather")
 
 
 def antdt_version() -> str:

@@ -50,6 +50,35 @@ __global__ void upload_small_kernel(SmallBlob blob, int n_words, uint32_t* dst) 
 }
 }  // namespace
 
+// Gather-rate probe: the plainest row gather there is.  A group of `dim/4` lanes owns one output
+// row and sums `per_out` input rows picked by consecutive entries of idx, one 16-byte vector per
+// lane and row, eight rows requested before the first add.  Timed on a matrix that fits L2 it
+// gives the rate at which the SMs can pull scattered rows out of L2, the ceiling of the
+// gathering kernels of the step once their rows are cache resident.
+template <int G>
+__global__ void __launch_bounds__(256)
+probe_gather_kernel(const float4* __restrict__ rows, uint32_t n_rows, const int32_t* __restrict__ idx,
+                    int64_t n_out, int per_out, float4* __restrict__ out) {
+  const int lg = threadIdx.x & (G - 1);
+  const int64_t o = ((int64_t)blockIdx.x * 256 + threadIdx.x) / G;
+  if (o >= n_out) return;
+  const int32_t* my = idx + o * per_out;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int j0 = 0; j0 < per_out; j0 += 8) {
+    float4 v[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      const uint32_t r = j0 + t < per_out ? (uint32_t)__ldg(my + j0 + t) : 0u;
+      v[t] = __ldg(rows + (size_t)(r < n_rows ? r : 0u) * G + lg);
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (j0 + t < per_out) { acc.x += v[t].x; acc.y += v[t].y; acc.z += v[t].z; acc.w += v[t].w; }
+    }
+  }
+  out[o * G + lg] = acc;
+}
+
 void upload_small(const void* host, size_t bytes, void* dev, cudaStream_t s) {
   const uint32_t* src = static_cast<const uint32_t*>(host);
   uint32_t* dst = static_cast<uint32_t*>(dev);
@@ -139,6 +168,31 @@ int32_t antdt_profile_get(int32_t idx, char* name, size_t name_cap, int64_t* lau
   if (launches) *launches = g_slots[idx].launches;
   if (total_ms) *total_ms = g_slots[idx].ms;
   return ANTDT_OK;
+}
+
+int32_t antdt_probe_gather(const float* rows, int64_t n_rows, int32_t dim, const int32_t* idx,
+                           int64_t n_out, int32_t per_out, float* out, void* stream) {
+  if (!rows || !idx || !out || n_rows < 1 || n_rows >= (1ll << 31) || n_out < 0 || per_out < 1 ||
+      n_out >= (1ll << 40) / 256)
+    return ANTDT_ERR_INVALID_ARG;
+  if (!antdt::aligned16(rows) || !antdt::aligned16(out)) return ANTDT_ERR_INVALID_ARG;
+  if (n_out == 0) return ANTDT_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  const float4* r4 = reinterpret_cast<const float4*>(rows);
+  float4* o4 = reinterpret_cast<float4*>(out);
+#define PROBE_CASE(G)                                                                            \
+  {                                                                                              \
+    const unsigned grid = (unsigned)((n_out * G + 255) / 256);                                   \
+    ANTDT_LAUNCH("probe_gather", antdt::probe_gather_kernel<G>, grid, 256, 0, s, r4,             \
+                 (uint32_t)n_rows, idx, n_out, per_out, o4);                                     \
+  }
+  if (dim == 16) PROBE_CASE(4)
+  else if (dim == 32) PROBE_CASE(8)
+  else if (dim == 64) PROBE_CASE(16)
+  else if (dim == 128) PROBE_CASE(32)
+  else return ANTDT_ERR_INVALID_ARG;
+#undef PROBE_CASE
+  return antdt::cuda_ok();
 }
 
 const char* antdt_version(void) { return "antdt-b200 0.1 (sm_100a)"; }

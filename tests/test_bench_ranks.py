@@ -37,3 +37,33 @@ def test_single_process_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5 and bench.sum_over_ranks(2.0) == 2.0
     bench.barrier()
+
+
+def test_reference_arm_runs_the_checker_only():
+    """`bench.py --impl reference` times the CPU checker and must not map the CUDA library: it
+    plans with the checker's own planner.  Run as a child process that lists what it mapped."""
+    import json
+    import subprocess
+    code = (
+        "import sys, json; sys.argv = ['bench.py', '--impl', 'reference', '--config', '1', "
+        "'--steps', '1', '--warmup', '0']; sys.path.insert(0, %r); import bench; bench.main(); "
+        "maps = open('/proc/self/maps').read(); "
+        "print(json.dumps({'antdt': 'libantdt' in maps, 'oracle': 'liboracle' in maps}))" % ROOT)
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="")
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env,
+                         timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    line, loaded = json.loads(lines[0]), json.loads(lines[1])
+    assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["cores"] == 1
+    assert line["cpu_baseline"]["cpu_model"] and line["cpu_baseline"]["cores_total"] >= 1
+    assert loaded == {"antdt": False, "oracle": True}
+    # its plan equals the library planner's (the two arms time the same batch)
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2404_09679_b200 import synth
+    w = synth.WORKLOADS[2]
+    a, b = bench.plan_all(w, 2), bench.plan_all_checker(w, 2)
+    for pa, pb in zip(a, b):
+        assert list(pa["batch_sizes"]) == pb["batch_sizes"] and list(pa["counts"]) == pb["counts"]
+        assert [tuple(r) for r in pa["ranges"]] == pb["ranges"]

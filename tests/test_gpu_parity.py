@@ -563,3 +563,14 @@ def test_bwd_extreme_row_ids_and_widest_rows():
                                         want["uniq_grads"], bsz)
     assert code == 0 and np.array_equal(aid, wid)
     G.close(agg, wagg, rtol=3e-5, atol=2e-6)
+
+
+def test_probe_gather_sums_the_rows_it_is_given():
+    rng = np.random.default_rng(91)
+    for D, per_out in ((16, 3), (32, 8), (64, 20), (128, 9)):
+        rows = rng.normal(size=(500, D)).astype(np.float32)
+        idx = rng.integers(0, 500, size=77 * per_out).astype(np.int32)
+        out = torch.full((77, D), float("nan"), device="cuda")
+        B.antdt_probe_gather(G.dev(rows), G.dev(idx), per_out, out)
+        want = rows.astype(np.float64)[idx.reshape(77, per_out)].sum(1)
+        G.close(out.cpu().numpy(), want)
