@@ -5,15 +5,15 @@
 //   expand    bag index of every occurrence (the sort's payload)
 //   sort      stable radix sort by row id inside each worker's range     (segsort.cu)
 //   runs      distinct rows, run starts, head bits, first run of each tile (segsort.cu)
-//   reduce    tile-parallel segmented sum of gathered d_pooled rows
-//   fixup     rows whose occurrences straddle tiles: ordered sum of the tiles' partials
+//   reduce    tile-parallel segmented sum of gathered d_pooled rows        (bwd_walk.cuh)
+//   fixup     rows whose occurrences leave a CTA's stretch of tiles: ordered sum of partials
 //
 // The reduction is balanced by occurrences, not by rows: a tile is 64 (small inputs: 16) consecutive
 // sorted occurrences whatever rows they belong to, so a row that holds 20% of a field's
 // occurrences costs its tiles no more than anyone else's.  Every sum has a fixed order (inside a
 // tile by sorted position, across tiles by tile index), no floating-point atomics anywhere.
 #include "segsort.cuh"
-#include "tile_reduce.cuh"
+#include "bwd_walk.cuh"
 
 namespace antdt {
 namespace {
@@ -23,7 +23,7 @@ size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 struct BwdLayout {
   SortLayout sort;
   size_t sort_ws, wso, occ_bounds, worker_b, keys_a, keys_b, vals_t, head_bits, tile_first,
-      head_part, tail_part, bytes;
+      head_part, tail_part, flags, tasks, bytes;
 };
 
 BwdLayout bwd_layout(int64_t nnz, int dim, int K, int tile_len) {
@@ -42,8 +42,11 @@ BwdLayout bwd_layout(int64_t nnz, int dim, int K, int tile_len) {
   L.vals_t = o;     o = align_up(o + 4 * n);
   L.head_bits = o;  o = align_up(o + 4 * head_bits_words((int64_t)n));
   L.tile_first = o; o = align_up(o + 4 * (n_tiles + 1));
-  L.head_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
-  L.tail_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
+  const size_t n_str = walk_stretches((int64_t)n, tile_len, dim);
+  L.head_part = o;  o = align_up(o + 4 * n_str * (size_t)dim);
+  L.tail_part = o;  o = align_up(o + 4 * n_str * (size_t)dim);
+  L.flags = o;      o = align_up(o + n_str);
+  L.tasks = o;      o = align_up(o + 4 * (2 * n_str + 4));
   L.bytes = o;
   return L;
 }
@@ -194,14 +197,18 @@ int32_t bwd_dedup_impl(
     t.K = K;
     t.out_cap = out_cap;
     t.out = uniq_grads;
-    t.head_part = (float*)(w8 + L.head_part);
-    t.tail_part = (float*)(w8 + L.tail_part);
+    WalkScratch tasks;
+    tasks.head_part = (float*)(w8 + L.head_part);
+    tasks.tail_part = (float*)(w8 + L.tail_part);
+    tasks.flags = (uint8_t*)(w8 + L.flags);
+    tasks.tasks = (int32_t*)(w8 + L.tasks);
     if (!arrival || arrival->n < 1) {
-      launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+      launch_bwd_walk(t, tasks, "seg_reduce_tiles", "seg_reduce_fixup", s);
     } else {
       // d_pooled is arriving piece by piece: a tile is walked as soon as the piece that holds
       // its last entry is there (the sort and the run detection above needed the ids only)
       const int64_t n_tiles = (nnz + tile_len - 1) / tile_len;
+      const int64_t tps = walk_tiles_per_stretch(dim);
       int64_t done = 0;  // tiles issued so far
       t.fixup = false;
       for (int c = 0; c < arrival->n; ++c) {
@@ -210,16 +217,17 @@ int32_t bwd_dedup_impl(
         if (c + 1 < arrival->n) {
           const int64_t e = arrival->entry_end[c];
           upto = e <= 0 ? 0 : (e >= nnz ? n_tiles : e / tile_len);  // tiles that end before entry e
+          if (upto < n_tiles) upto = upto / tps * tps;              // a launch walks whole stretches
         }
         if (upto <= done) continue;
         t.tile_begin = done;
         t.tile_end = upto;
-        launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+        launch_bwd_walk(t, tasks, "seg_reduce_tiles", "seg_reduce_fixup", s);
         done = upto;
       }
       t.walk = false;
       t.fixup = true;
-      launch_tile_reduce<false>(t, "seg_reduce_tiles", "seg_reduce_fixup", s);
+      launch_bwd_walk(t, tasks, "seg_reduce_tiles", "seg_reduce_fixup", s);
     }
   }
   return cuda_ok();
