@@ -614,7 +614,9 @@ def run_ours(args):
         "e2e": None if args.no_e2e else {
             "value": e2e_samples / (e2e_ms * 1e-3), "unit": UNIT,
             "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-            "ms_per_step": e2e_ms / K_steps},
+            "ms_per_step": e2e_ms / K_steps,
+            "how": "antdt_bsp_step_host, two staging sets alternated: the copies of step s+1 run "
+                   "under the kernels of step s; the host reads every step's results"},
         "gpu_launches": launches,
         "roofline": roof,
         "step_algorithmic_GB": round(sb / 1e9, 3),
@@ -664,67 +666,48 @@ def measure_l2_gather(B, dev, row_bytes, stream, _cache={}):
 
 def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream):
     """K steps through antdt_bsp_step_host; every step copies its inputs from page-locked host
-    memory and its results back, and the host waits for them."""
-    def pin(t):
-        return t.cpu().pin_memory()
+    memory and its results back, and the host reads every step's results.  Two staging sets are
+    alternated so that the copies of step s+1 run under the kernels of step s; the host reads step
+    s's results while step s+1 is in flight."""
+    from paper_2404_09679_b200.step import HostStaging, HostStep
 
-    host = [dict(ids=pin(b["ids"]), off=pin(b["off"]), dY=pin(b["dY"]),
-                 dense=None if b["dense"] is None else pin(b["dense"])) for b in batches]
+    def pin(t):
+        return None if t is None else t.cpu().pin_memory()
+
+    host = [dict(ids=pin(b["ids"]), off=pin(b["off"]), dY=pin(b["dY"]), dense=pin(b["dense"]))
+            for b in batches]
     max_nnz = max(b["ids"].numel() for b in batches)
     max_bags = max(b["off"].numel() - 1 for b in batches)
-    d_ids = torch.empty(max_nnz, dtype=torch.int32, device=dev)
-    d_off = torch.empty(max_bags + 1, dtype=torch.int64, device=dev)
-    d_dY = torch.empty(max_bags, w.D, dtype=torch.float32, device=dev)
-    d_dense = torch.empty(w.K, w.dense_n, dtype=torch.float32, device=dev) if w.dense_n else None
-    h_pooled = torch.empty(max_bags, w.D, dtype=torch.float32).pin_memory()
-    h_dense_out = torch.empty(w.dense_n, dtype=torch.float32).pin_memory() if w.dense_n else None
-    h_n_agg = torch.zeros(1, dtype=torch.int64).pin_memory()
-    h_status = torch.zeros(1, dtype=torch.int32).pin_memory()
-    keep = []
-
-    def desc_for(j, step):
-        b, h = batches[j], host[j]
-        wso = (C.c_int64 * (w.K + 1))(*[int(x) for x in b["wso"]])
-        bsz = (C.c_int64 * w.K)(*[int(x) for x in b["counts"]])
-        keep[:] = [wso, bsz]
-        p = lambda t: None if t is None else t.data_ptr()  # noqa: E731
-        d = B.StepDesc()
-        d.table, d.dtype, d.n_rows, d.dim = p(table), (B.BF16 if table.dtype == torch.bfloat16 else B.F32), w.V, w.D
-        d.state0, d.state1 = p(state0), p(state1)
-        d.opt, d.lr, d.eps, d.beta1, d.beta2, d.step = oc.opt, oc.lr, oc.eps, oc.beta1, oc.beta2, step
-        d.h_row_ids, d.nnz = p(h["ids"]), b["ids"].numel()
-        d.h_bag_offsets, d.n_bags, d.bags_per_sample = p(h["off"]), b["off"].numel() - 1, w.F
-        d.h_d_pooled, d.h_dense_grads, d.dense_n = p(h["dY"]), p(h["dense"]), w.dense_n
-        d.n_workers = w.K
-        d.worker_sample_offsets = C.cast(wso, C.c_void_p)
-        d.batch_sizes = C.cast(bsz, C.c_void_p)
-        d.d_row_ids, d.d_bag_offsets, d.d_pooled_out, d.d_d_pooled = p(d_ids), p(d_off), p(buf.pooled), p(d_dY)
-        d.d_dense_grads, d.d_dense_out = p(d_dense), p(buf.dense_out)
-        d.d_uniq_ids, d.d_worker_uniq_offsets = p(buf.uniq_ids), p(buf.worker_uniq_offsets)
-        d.d_seg_offsets, d.d_sorted_occ, d.d_uniq_grads = p(buf.seg_offsets), p(buf.sorted_occ), p(buf.uniq_grads)
-        d.uniq_cap = buf.uniq_cap
-        d.d_agg_ids, d.d_agg_grads, d.d_n_agg, d.agg_cap = p(buf.agg_ids), p(buf.agg_grads), p(buf.n_agg), buf.agg_cap
-        d.ws, d.ws_bytes, d.d_status = p(buf.ws), buf.ws.numel(), p(buf.status)
-        d.h_pooled, d.h_dense_out, d.h_n_agg, d.h_status = p(h_pooled), p(h_dense_out), p(h_n_agg), p(h_status)
-        return d
-
+    sets = [HostStaging(w.D, w.K, max_nnz, max_bags, w.dense_n, dev) for _ in range(2)]
+    hs = HostStep(buf, table, state0, state1, oc, w.K)
     n_b = len(batches)
+
+    def issue(s, step, idle):
+        j = s % n_b
+        b, h, st = batches[j], host[j], sets[s % 2]
+        hs.run(st, step, h["ids"], h["off"], w.F, h["dY"], b["wso"], b["counts"], h["dense"],
+               stream=stream, staging_idle=idle)
+        return st
+
+    def collect(st):
+        st.done.synchronize()                             # the caller reads the step's results
+        assert int(st.h_status[0]) == 0 and int(st.h_n_agg[0]) > 0
+
     step0 = 10_000
     for s in range(min(W, 3)):
-        B.antdt_bsp_step_host(desc_for(s % n_b, step0 + s), stream)
-        torch.cuda.synchronize()
-        assert int(h_status[0]) == 0
+        collect(issue(s, step0 + s, False))
     barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    samples = 0
+    samples, pending = 0, None
     for s in range(K_steps):
-        j = s % n_b
-        B.antdt_bsp_step_host(desc_for(j, step0 + 3 + s), stream)
-        stream.synchronize()                              # the caller reads the step's results
-        assert int(h_status[0]) == 0 and int(h_n_agg[0]) > 0
-        samples += sum(batches[j]["counts"])
+        st = issue(s, step0 + 3 + s, True)                # its set was collected two steps ago
+        if pending is not None:
+            collect(pending)
+        pending = st
+        samples += sum(batches[s % n_b]["counts"])
+    collect(pending)
     e1.record(stream)
     torch.cuda.synchronize()
     barrier()

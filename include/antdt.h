@@ -349,9 +349,18 @@ int32_t antdt_dense_opt_update(float* params, const float* grad, int64_t n, int3
  * buffers, runs fwd, bwd_dedup, aggregate and update in order on `stream`, and copies the
  * results (pooled, dense_out, n_agg, status) back.  The copies run on two internal side
  * streams (created on the first call on a device) so that they overlap the kernels; `stream`
- * waits for all of them before the call's work on it ends, so synchronising `stream` is enough.
- * Host buffers should be page-locked for the copies to overlap.  Every pointer of the
- * descriptor is described beside its field. */
+ * waits for all of them before the call's work on it ends, so synchronising `stream` (or an
+ * event recorded on it after the call) is enough.  Host buffers should be page-locked for the
+ * copies to overlap.  Every pointer of the descriptor is described beside its field.
+ *
+ * Two steps in flight.  By default the input copies wait for everything issued earlier on
+ * `stream`, because the staging buffers may still be in use by it.  A caller that keeps TWO
+ * sets of the buffers the copies touch - d_row_ids, d_bag_offsets, d_d_pooled, d_dense_grads,
+ * d_pooled_out, d_dense_out, d_n_agg, d_status and the h_* outputs - and alternates them sets
+ * staging_idle = 1: the copies of step s+1 then start at once and run under the kernels of step
+ * s (the kernels themselves stay in order on `stream`; table, state, workspace and the other
+ * intermediates are shared).  The caller records an event on `stream` after each call and waits
+ * for that event before it reads the step's h_* results or reuses its set. */
 typedef struct {
   /* model state, device resident */
   void* table; int32_t dtype; int64_t n_rows; int32_t dim;
@@ -378,6 +387,7 @@ typedef struct {
   float* h_pooled;                      /* host [n_bags, dim]                              */
   float* h_dense_out;                   /* host [dense_n] or NULL                          */
   int64_t* h_n_agg; int32_t* h_status;  /* one element each                                */
+  int32_t staging_idle;                 /* antdt_bsp_step_host only, see above; 0 = wait     */
 } antdt_step_desc;
 int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream);
 /* The same step for a batch that already sits in device memory: the d_row_ids, d_bag_offsets,

@@ -83,7 +83,7 @@ class StepDesc(C.Structure):
         ("agg_cap", C.c_int64),
         ("ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("d_status", C.c_void_p),
         ("h_pooled", C.c_void_p), ("h_dense_out", C.c_void_p), ("h_n_agg", C.c_void_p),
-        ("h_status", C.c_void_p),
+        ("h_status", C.c_void_p), ("staging_idle", C.c_int32),
     ]
 
 

@@ -57,10 +57,14 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
   if (!ss) return ANTDT_ERR_CUDA;
 
 #define CK(x) do { if ((x) != cudaSuccess) return ANTDT_ERR_CUDA; } while (0)
-  // inputs: everything earlier on the caller's stream first (the staging buffers are reused)
-  CK(cudaEventRecord(ss->start, s));
-  CK(cudaStreamWaitEvent(ss->in, ss->start, 0));
-  CK(cudaStreamWaitEvent(ss->out, ss->start, 0));
+  // inputs: everything earlier on the caller's stream first (the staging buffers are reused),
+  // unless the caller vouches that this descriptor's set is idle: then the copies start at once
+  // and run under whatever the stream is still computing (the previous step)
+  if (!d->staging_idle) {
+    CK(cudaEventRecord(ss->start, s));
+    CK(cudaStreamWaitEvent(ss->in, ss->start, 0));
+    CK(cudaStreamWaitEvent(ss->out, ss->start, 0));
+  }
   CK(cudaMemcpyAsync(d->d_bag_offsets, d->h_bag_offsets, 8 * ((size_t)d->n_bags + 1),
                      cudaMemcpyHostToDevice, ss->in));
   if (d->nnz > 0)

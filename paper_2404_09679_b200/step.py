@@ -113,3 +113,59 @@ class DeviceStep:
             B.antdt_bsp_step_graph(d, stream)
         else:
             B.antdt_bsp_step_device(d, stream)
+
+
+class HostStaging:
+    """One set of the buffers antdt_bsp_step_host copies through: device staging for the inputs,
+    device and page-locked host buffers for the results.  A caller that keeps two of these and
+    alternates them may have two steps in flight (staging_idle in the descriptor)."""
+
+    def __init__(self, dim: int, n_workers: int, max_nnz: int, max_bags: int, dense_n: int = 0,
+                 device="cuda"):
+        dev = torch.device(device)
+        i32, i64, f32 = torch.int32, torch.int64, torch.float32
+        self.d_row_ids = torch.empty(max(max_nnz, 1), dtype=i32, device=dev)
+        self.d_bag_offsets = torch.empty(max_bags + 1, dtype=i64, device=dev)
+        self.d_d_pooled = torch.empty(max(max_bags, 1), dim, dtype=f32, device=dev)
+        self.d_dense_grads = torch.empty(n_workers, dense_n, dtype=f32, device=dev) if dense_n else None
+        self.d_pooled_out = torch.empty(max(max_bags, 1), dim, dtype=f32, device=dev)
+        self.d_dense_out = torch.empty(dense_n, dtype=f32, device=dev) if dense_n else None
+        self.d_n_agg = torch.zeros(1, dtype=i64, device=dev)
+        self.d_status = torch.zeros(1, dtype=i32, device=dev)
+        self.h_pooled = torch.empty(max(max_bags, 1), dim, dtype=f32).pin_memory()
+        self.h_dense_out = torch.empty(dense_n, dtype=f32).pin_memory() if dense_n else None
+        self.h_n_agg = torch.zeros(1, dtype=i64).pin_memory()
+        self.h_status = torch.zeros(1, dtype=i32).pin_memory()
+        self.done = torch.cuda.Event()   # recorded by HostStep.run after the call
+
+
+class HostStep:
+    """antdt_bsp_step_host for a model state and a buffer set; `run` fills the descriptor for one
+    batch given as page-locked host tensors and one HostStaging set."""
+
+    def __init__(self, buf: StepBuffers, table, state0, state1, oc: OptConfig, n_workers: int):
+        import ctypes as C
+        self._inner = DeviceStep(buf, table, state0, state1, oc, n_workers)
+        self._C = C
+
+    def run(self, st: HostStaging, step: int, h_row_ids, h_bag_offsets, bags_per_sample: int,
+            h_d_pooled, worker_sample_offsets: Sequence[int], batch_sizes: Sequence[int],
+            h_dense_grads=None, stream=None, staging_idle: bool = False):
+        d = self._inner.desc
+        p = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        d.step = step
+        d.h_row_ids, d.nnz = p(h_row_ids), h_row_ids.numel()
+        d.h_bag_offsets, d.n_bags = p(h_bag_offsets), h_bag_offsets.numel() - 1
+        d.bags_per_sample = bags_per_sample
+        d.h_d_pooled, d.h_dense_grads = p(h_d_pooled), p(h_dense_grads)
+        d.dense_n = 0 if h_dense_grads is None else h_dense_grads.shape[1]
+        self._inner._wso[:] = [int(x) for x in worker_sample_offsets]
+        self._inner._bsz[:] = [int(x) for x in batch_sizes]
+        d.d_row_ids, d.d_bag_offsets, d.d_d_pooled = p(st.d_row_ids), p(st.d_bag_offsets), p(st.d_d_pooled)
+        d.d_dense_grads, d.d_pooled_out, d.d_dense_out = p(st.d_dense_grads), p(st.d_pooled_out), p(st.d_dense_out)
+        d.d_n_agg, d.d_status = p(st.d_n_agg), p(st.d_status)
+        d.h_pooled, d.h_dense_out = p(st.h_pooled), p(st.h_dense_out)
+        d.h_n_agg, d.h_status = p(st.h_n_agg), p(st.h_status)
+        d.staging_idle = 1 if staging_idle else 0
+        B.antdt_bsp_step_host(d, stream)
+        st.done.record(stream if stream is not None else torch.cuda.current_stream())

@@ -122,3 +122,59 @@ def test_single_call_device_step_equals_the_four_calls():
         assert torch.equal(buf_b.agg_grads[:na], buf_a.agg_grads[:na])
         assert torch.equal(buf_b.dense_out, buf_a.dense_out)
         assert torch.equal(t_b, t_a) and torch.equal(s0_b, s0_a) and torch.equal(s1_b, s1_a)
+
+
+def test_two_host_steps_in_flight_equal_one_at_a_time():
+    """Two staging sets alternated with staging_idle: the copies of a step run under the kernels
+    of the step before it.  Results (host outputs of every step, table and state at the end) must
+    be bit-identical to the same steps issued one at a time."""
+    from paper_2404_09679_b200.step import HostStaging, HostStep
+    w = synth.WORKLOADS[4].scaled(B=4096, V=400_000)
+    n_steps = 5
+    plans = plan_steps(w, n_steps)
+    bm = synth.BatchMaker(w, "cuda")
+    table0 = bm.table()
+    oc = OptConfig(B.OPTS[w.opt], w.lr, w.eps, w.beta1, w.beta2)
+    batches = [make_batch(bm, plans[s], s) for s in range(n_steps)]
+    pin = lambda t: None if t is None else t.cpu().pin_memory()  # noqa: E731
+    host = [dict(ids=pin(b["row_ids"]), off=pin(b["bag_offsets"]), dY=pin(b["d_pooled"]),
+                 dense=pin(b["dense"])) for b in batches]
+    max_nnz = max(b["row_ids"].numel() for b in batches)
+    max_bags = max(b["bag_offsets"].numel() - 1 for b in batches)
+    stream = torch.cuda.Stream()
+    results = {}
+    for mode in ("serial", "overlap"):
+        table = table0.clone()
+        s0 = torch.zeros(w.V, w.D, device="cuda")
+        buf = StepBuffers(w.D, w.K, max_nnz, max_bags, w.dense_n)
+        sets = [HostStaging(w.D, w.K, max_nnz, max_bags, w.dense_n) for _ in range(2)]
+        hs = HostStep(buf, table, s0, None, oc, w.K)
+        torch.cuda.synchronize()
+        outs, pending = [], None
+
+        def collect(st, s):
+            st.done.synchronize()
+            assert int(st.h_status[0]) == 0
+            nb = batches[s]["bag_offsets"].numel() - 1
+            outs.append((int(st.h_n_agg[0]), st.h_pooled[:nb].clone()))
+
+        for s in range(n_steps):
+            b, h = batches[s], host[s]
+            st = sets[s % 2]
+            hs.run(st, s + 1, h["ids"], h["off"], w.F, h["dY"], b["wso"].tolist(), b["counts"].tolist(),
+                   h["dense"], stream=stream, staging_idle=(mode == "overlap"))
+            if mode == "serial":
+                collect(st, s)
+            else:
+                if pending is not None:
+                    collect(*pending)
+                pending = (st, s)
+        if pending is not None:
+            collect(*pending)
+        torch.cuda.synchronize()
+        results[mode] = (outs, table.view(torch.int16).clone(), s0.clone())
+    (o_a, t_a, s_a), (o_b, t_b, s_b) = results["serial"], results["overlap"]
+    assert [n for n, _ in o_a] == [n for n, _ in o_b]
+    for (_, pa), (_, pb) in zip(o_a, o_b):
+        assert torch.equal(pa, pb)
+    assert torch.equal(t_a, t_b) and torch.equal(s_a, s_b)
