@@ -268,15 +268,19 @@ def algorithmic_bytes(w, nnz, n_bags, sum_u, u):
         "expand_bags": 8 * (n_bags + 1) + 4 * nnz,
         "seg_reduce_tiles": 4 * nnz + nnz // 8 + nnz * D * 4 + sum_u * D * 4,
         "agg_reduce": sum_u * (4 * D + 4) + u * (4 * D + 8),
+        # one pass: contributions in, table and state in and out; no aggregated gradient in between
+        "agg_update": sum_u * (4 * D + 4) + u * 8 + 2 * u * D * ew + 2 * S * u * D * 4,
         "sparse_adagrad": u * (4 + 4 * D) + 2 * u * D * ew + 2 * S * u * D * 4,
         "sparse_adam": u * (4 + 4 * D) + 2 * u * D * ew + 2 * S * u * D * 4,
         "dense_wsum": (w.K + 1) * w.dense_n * 4,
     }
 
 
-def step_bytes(w, nnz, n_bags, sum_u, u, passes_bwd, passes_agg):
+def step_bytes(w, nnz, n_bags, sum_u, u, passes_bwd, passes_agg, fused=False):
     b = algorithmic_bytes(w, nnz, n_bags, sum_u, u)
     upd = b["sparse_adam"] if w.opt == "adam" else b["sparse_adagrad"]
+    if fused and w.K <= 32:   # the one-pass server step: no aggregated gradient in between
+        upd = b["agg_update"] - b["agg_reduce"]
     sort = passes_bwd * (b["radix_hist"] + b["radix_scatter"]) + b["runs_count"] + b["runs_emit"]
     if w.K <= 32:       # the aggregation's merge order comes from the range pass, not a sort
         sort += b["agg_range_count"] + b["agg_range_emit"]
@@ -435,7 +439,8 @@ def run_ours(args):
     buf = StepBuffers(w.D, w.K, max_nnz, max_bags, w.dense_n, uniq_cap=cap, agg_cap=cap, device=dev)
 
     dds = B.Dds(w.n_samples, w.B, w.M, w.K)                # the live planner of the timed loop
-    dstep = DeviceStep(buf, table, state0, state1, oc, w.K)  # the four device calls behind one C call
+    # the device calls behind one C call; --fuse-update: aggregate and update in one pass
+    dstep = DeviceStep(buf, table, state0, state1, oc, w.K, fuse_update=args.fuse_update)
 
     # Launch form of the timed steps.  A step is 30-40 launches; on the small configurations
     # they, not the kernels, are the step time, so there the step is replayed as one CUDA graph.
@@ -512,7 +517,8 @@ def run_ours(args):
     if args.no_e2e:
         e2e = {"ms": float("nan"), "samples": 0, "h2d": 0, "d2h": 0}
     else:
-        e2e = run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream)
+        e2e = run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream,
+                      args.fuse_update)
     e2e_ms = max_over_ranks(e2e["ms"], dev)
     e2e_samples = sum_over_ranks(float(e2e["samples"]), dev)
 
@@ -595,7 +601,7 @@ def run_ours(args):
         roof["l2_gather"] = l2.get(top)
     rowbits = max(1, (w.V - 1).bit_length())
     passes = -(-rowbits // 9)
-    sb = step_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen, passes, passes)
+    sb = step_bytes(w, int(nnz_avg), int(bags_avg), sum_u_seen, u_seen, passes, passes, args.fuse_update)
     line = {
         "metric": METRIC, "value": samples / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": K_steps, "warmup": W, "ms_per_step": ms / K_steps, "higher_is_better": True,
@@ -608,6 +614,8 @@ def run_ours(args):
                          "126 MB L2", "batches_rotated": n_batches,
                    "launch": ("one CUDA graph per step (antdt_bsp_step_graph)" if use_graph
                               else "plain launches (antdt_bsp_step_device)"),
+                   "server_step": ("one pass (antdt_aggregate_update)" if args.fuse_update
+                                   else "aggregate, then update"),
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"],
                    "samples": clk["samples"], "extra_warmup_steps": extra},
@@ -664,7 +672,7 @@ def measure_l2_gather(B, dev, row_bytes, stream, _cache={}):
     return _cache[row_bytes]
 
 
-def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream):
+def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stream, fuse_update=False):
     """K steps through antdt_bsp_step_host; every step copies its inputs from page-locked host
     memory and its results back, and the host reads every step's results.  Two staging sets are
     alternated so that the copies of step s+1 run under the kernels of step s; the host reads step
@@ -679,7 +687,7 @@ def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stre
     max_nnz = max(b["ids"].numel() for b in batches)
     max_bags = max(b["off"].numel() - 1 for b in batches)
     sets = [HostStaging(w.D, w.K, max_nnz, max_bags, w.dense_n, dev) for _ in range(2)]
-    hs = HostStep(buf, table, state0, state1, oc, w.K)
+    hs = HostStep(buf, table, state0, state1, oc, w.K, fuse_update)
     n_b = len(batches)
 
     def issue(s, step, idle):
@@ -780,6 +788,9 @@ def main():
                          "for the launch-bound configs 1 and 2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--fuse-update", action="store_true",
+                    help="server step through antdt_aggregate_update (aggregated gradients not "
+                         "materialised)")
     ap.add_argument("--no-l2-probe", action="store_true",
                     help="skip the L2 gather-rate probe (profiling runs)")
     ap.add_argument("--scale", type=float, default=1.0,

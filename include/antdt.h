@@ -276,8 +276,9 @@ int32_t antdt_embbag_bwd_dedup_static(const int32_t* row_ids, int64_t nnz,
  * hold a row contributes nothing; summed in ascending worker order.  Dense part: the same
  * weights over K dense vectors.  Either part may be NULL.  Every worker's list must ascend
  * strictly (what antdt_embbag_bwd_dedup writes does); a list of up to 32 workers that repeats
- * ids so often that a stretch of 4096 consecutive row ids holds more entries than K times
- * its width raises BAD_OFFSETS in dev_status and that stretch is left out of the result.
+ * ids so often that a stretch of 4096 consecutive row ids (8192 for tables beyond 2^30 rows or
+ * inputs that hit the table sparsely) holds more entries than K times its width raises
+ * BAD_OFFSETS in dev_status and that stretch is left out of the result.
  *   batch_sizes host [K] int64: the b_i actually served this step (counts), sum > 0. */
 typedef struct {
   int32_t dim;
@@ -335,6 +336,23 @@ int32_t antdt_sparse_opt_update(void* table, int32_t dtype, int64_t n_rows, int3
                                 float eps, float beta1, float beta2, int64_t step, float* state0,
                                 float* state1, int32_t* dev_status, void* stream);
 
+/* Aggregation and sparse update in one call (Section II: the servers aggregate the local
+ * gradients and update the parameters - one step of theirs): the result in table / state0 /
+ * state1 is that of antdt_weighted_aggregate followed by antdt_sparse_opt_update with the same
+ * arguments (opt: ANTDT_OPT_ADAGRAD or ANTDT_OPT_ADAM), up to the rounding order of the weighted
+ * sums (ascending worker, one fused multiply-add per contribution).  With up to 32 workers it is
+ * ONE pass over the aggregated rows: each row's contributions are summed by the lane group that
+ * then applies them, so the aggregated gradients are neither written nor read back;
+ * sp->agg_grads may then be NULL (not materialised) - if given it is filled as usual.  agg_ids,
+ * n_agg and the dense part are produced as by antdt_weighted_aggregate.  With more than 32
+ * workers the two steps run one after the other and sp->agg_grads is required.
+ * Workspace: antdt_weighted_aggregate_workspace_bytes.  Errors as the two calls'. */
+int32_t antdt_aggregate_update(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                               const int64_t* batch_sizes, int32_t n_workers, void* table,
+                               int32_t dtype, int32_t opt, float lr, float eps, float beta1,
+                               float beta2, int64_t step, float* state0, float* state1, void* ws,
+                               size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* Server update of the DENSE parameters (Section II: after aggregating, the servers update
  * the parameters): the element-wise Adagrad / Adam formulas above on a dense fp32 vector, with
  * the gradient antdt_weighted_aggregate's dense part produced.  Every element is touched.
@@ -388,6 +406,8 @@ typedef struct {
   float* h_dense_out;                   /* host [dense_n] or NULL                          */
   int64_t* h_n_agg; int32_t* h_status;  /* one element each                                */
   int32_t staging_idle;                 /* antdt_bsp_step_host only, see above; 0 = wait     */
+  int32_t fuse_update;                  /* 1: aggregate and update through                   */
+                                        /* antdt_aggregate_update, d_agg_grads not written   */
 } antdt_step_desc;
 int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream);
 /* The same step for a batch that already sits in device memory: the d_row_ids, d_bag_offsets,

@@ -33,7 +33,7 @@ EXPORTS = [
     "antdt_embbag_bwd_dedup",
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
-    "antdt_weighted_aggregate_backup",
+    "antdt_weighted_aggregate_backup", "antdt_aggregate_update",
     "antdt_sparse_opt_update", "antdt_dense_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_bsp_step_graph", "antdt_bsp_step_graph_reset",
     "antdt_read_status", "antdt_launch_count",
     "antdt_profile_enable", "antdt_profile_kernels", "antdt_profile_get", "antdt_probe_gather",
@@ -83,7 +83,7 @@ class StepDesc(C.Structure):
         ("agg_cap", C.c_int64),
         ("ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("d_status", C.c_void_p),
         ("h_pooled", C.c_void_p), ("h_dense_out", C.c_void_p), ("h_n_agg", C.c_void_p),
-        ("h_status", C.c_void_p), ("staging_idle", C.c_int32),
+        ("h_status", C.c_void_p), ("staging_idle", C.c_int32), ("fuse_update", C.c_int32),
     ]
 
 
@@ -130,6 +130,9 @@ def lib() -> C.CDLL:
         L.antdt_weighted_aggregate.argtypes = [P, P, P, I32, P, SZ, P, P]
         L.antdt_weighted_aggregate_backup.argtypes = [P, P, P, P, I32, P, SZ, P, P]
         L.antdt_weighted_aggregate_backup.restype = I32
+        L.antdt_aggregate_update.argtypes = [P, P, P, I32, P, I32, I32, C.c_float, C.c_float, C.c_float,
+                                             C.c_float, I64, P, P, P, SZ, P, P]
+        L.antdt_aggregate_update.restype = I32
         L.antdt_sparse_opt_update.argtypes = [P, I32, I64, I32, P, P, P, I64, I32, F, F, F, F, I64,
                                               P, P, P, P]
         L.antdt_dense_opt_update.argtypes = [P, P, I64, I32, F, F, F, F, I64, P, P, P]
@@ -391,6 +394,28 @@ def antdt_weighted_aggregate(batch_sizes: Sequence[int], ws, *, n_rows: int = 0,
         C.byref(sp) if sp else None, C.byref(dp) if dp else None, _i64s(batch_sizes), K, _dp(ws),
         ws.numel() * ws.element_size(), _dp(dev_status), _stream(stream)),
         "antdt_weighted_aggregate")
+
+
+def antdt_aggregate_update(batch_sizes: Sequence[int], ws, table, opt: int, lr: float, eps: float,
+                           beta1: float, beta2: float, step: int, state0, state1=None, *,
+                           uniq_ids, worker_uniq_offsets, uniq_grads, agg_ids, n_agg, agg_grads=None,
+                           dense_grads=None, dense_out=None, dev_status=None, stream=None):
+    """antdt_weighted_aggregate + antdt_sparse_opt_update in one call (one pass for <= 32 workers);
+    agg_grads=None: the aggregated gradients are not materialised."""
+    K = len(batch_sizes)
+    V, D = table.shape
+    sp = SparsePart(D, V, uniq_ids.data_ptr(), worker_uniq_offsets.data_ptr(), uniq_grads.data_ptr(),
+                    uniq_grads.shape[0], agg_ids.data_ptr(),
+                    None if agg_grads is None else agg_grads.data_ptr(), n_agg.data_ptr(),
+                    agg_ids.shape[0])
+    dp = None
+    if dense_grads is not None:
+        dp = DensePart(dense_grads.data_ptr(), dense_grads.shape[1], dense_grads.stride(0),
+                       dense_out.data_ptr())
+    _check(lib().antdt_aggregate_update(
+        C.byref(sp), C.byref(dp) if dp else None, _i64s(batch_sizes), K, _dp(table), _dtype_code(table),
+        opt, lr, eps, beta1, beta2, step, _dp(state0), _dp(state1), _dp(ws),
+        ws.numel() * ws.element_size(), _dp(dev_status), _stream(stream)), "antdt_aggregate_update")
 
 
 def antdt_sparse_opt_update(table, ids, grads, n_ids_dev, opt: int, lr: float, eps: float,

@@ -245,7 +245,8 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
                   const int64_t* __restrict__ wuo, int K, int64_t P, int r_log2, int64_t n_rows,
                   uint32_t dropped, const int64_t* __restrict__ base, int32_t* __restrict__ agg_ids,
                   int64_t out_cap, uint32_t* __restrict__ src, uint32_t* head_bits,
-                  int32_t* __restrict__ tile_first, int tile_shift, int32_t* status) {
+                  int32_t* __restrict__ tile_first, int tile_shift, uint32_t* __restrict__ row_start,
+                  int32_t* status) {
   extern __shared__ __align__(16) unsigned char ra_smem[];
   const int R = 1 << r_log2;
   const int nW = R / 32;  // presence words: at most 256 = one per thread
@@ -321,7 +322,10 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
                    const int64_t dest = pc.before + (int64_t)first_c[t] + slot;
                    const int64_t u = u0 + t;
                    src[dest] = (uint32_t)j;
-                   if (slot == 0 && u < out_cap) agg_ids[u] = (int32_t)id;
+                   if (slot == 0 && u < out_cap) {
+                     agg_ids[u] = (int32_t)id;
+                     if (row_start) row_start[u] = (uint32_t)dest;  // the row's first merge slot
+                   }
                    if ((dest & tile_mask) == 0) tile_first[dest >> tile_shift] = (int32_t)u;
                  });
 }
@@ -358,10 +362,10 @@ void range_prepare_device() {
 void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t in_cap, int64_t n_rows,
                        int K, uint32_t dropped_bits, int32_t* agg_ids, int64_t* n_agg, int64_t out_cap,
                        int64_t* wuo_out, int64_t* n_entries, uint32_t* src, uint32_t* head_bits,
-                       int32_t* tile_first, int tile, char* ws, const RangeLayout& L, int32_t* status,
-                       cudaStream_t s) {
+                       int32_t* tile_first, int tile, uint32_t* row_start, char* ws, const RangeLayout& L,
+                       int32_t* status, cudaStream_t s) {
   range_prepare_device();
-  const int r_log2 = range_log2(n_rows);
+  const int r_log2 = range_log2(n_rows, in_cap);
   const int64_t P = (n_rows + ((int64_t)1 << r_log2) - 1) >> r_log2;  // <= kRangeMaxRanges
   int32_t* bnd = (int32_t*)(ws + L.bnd);
   int32_t* distinct = (int32_t*)(ws + L.distinct);
@@ -381,7 +385,7 @@ void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t i
   cudaMemsetAsync(tile_first, 0, 4 * ((size_t)((in_cap + tile - 1) >> tile_shift) + 1), s);
   ANTDT_LAUNCH("agg_range_emit", range_emit_kernel, (unsigned)P, kRaThreads, emit_smem(r_log2, K), s,
                uniq_ids, bnd, wuo_out, K, P, r_log2, n_rows, dropped_bits, base, agg_ids, out_cap, src,
-               head_bits, tile_first, tile_shift, status);
+               head_bits, tile_first, tile_shift, row_start, status);
 }
 
 }  // namespace antdt

@@ -18,9 +18,13 @@ constexpr int kRangeLog2 = 12;              // 4096 row ids per range (measured 
 constexpr int kRangeMaxLog2 = 13;           // 8192 for tables beyond 2^30 rows (bounds the scratch)
 constexpr int64_t kRangeMaxRanges = (int64_t)1 << (31 - kRangeMaxLog2);  // n_rows < 2^31
 
-// log2 of the range width
-inline int range_log2(int64_t n_rows) {
-  return n_rows > ((int64_t)kRangeMaxRanges << kRangeLog2) ? kRangeMaxLog2 : kRangeLog2;
+// log2 of the range width.  The wide ranges also serve an input that is sparse in the table
+// (fewer than 64 entries per narrow range on average): a range CTA's cost is mostly its fixed part
+// then, so half as many CTAs finish sooner.
+inline int range_log2(int64_t n_rows, int64_t in_cap) {
+  if (n_rows > ((int64_t)kRangeMaxRanges << kRangeLog2)) return kRangeMaxLog2;
+  const int64_t narrow = (n_rows + ((int64_t)1 << kRangeLog2) - 1) >> kRangeLog2;
+  return in_cap < 64 * narrow ? kRangeMaxLog2 : kRangeLog2;
 }
 
 struct RangeLayout {
@@ -43,10 +47,11 @@ void range_prepare_device();
 //                       slots ordered by (row id, worker)
 //   head_bits           bit i set iff slot i is the first contribution of its row (zeroed here)
 //   tile_first          index into agg_ids of the row that slot t*tile belongs to
+//   row_start [out_cap] merge slot of the first contribution of each row of agg_ids, or nullptr
 void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t in_cap, int64_t n_rows,
                        int K, uint32_t dropped_bits, int32_t* agg_ids, int64_t* n_agg, int64_t out_cap,
                        int64_t* wuo_out, int64_t* n_entries, uint32_t* src, uint32_t* head_bits,
-                       int32_t* tile_first, int tile, char* ws, const RangeLayout& L, int32_t* status,
-                       cudaStream_t s);
+                       int32_t* tile_first, int tile, uint32_t* row_start, char* ws, const RangeLayout& L,
+                       int32_t* status, cudaStream_t s);
 
 }  // namespace antdt

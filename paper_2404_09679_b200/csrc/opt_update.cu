@@ -5,49 +5,12 @@
 // bf16), widened to fp32, updated and stored back round-to-nearest-even.  The ids ascend, so
 // the row accesses sweep the table forward.  Division and square root are the IEEE-rounded
 // ones (no fast-math).
-#include "common.cuh"
+#include "opt_math.cuh"
 
 namespace antdt {
 namespace {
 
 constexpr int kOptThreads = 256;
-
-struct OptParams {
-  float lr, eps, beta1, beta2;
-  float omb1, omb2;  // 1 - beta
-  float bc1, bc2;    // 1 - beta^t
-};
-
-__device__ __forceinline__ float4 load_row4(const void* table, bool bf16, size_t elem) {
-  if (bf16) {
-    const uint2 v = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(table) + elem);
-    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u),
-                       __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
-  }
-  return *reinterpret_cast<const float4*>(static_cast<const float*>(table) + elem);
-}
-
-__device__ __forceinline__ void store_row4(void* table, bool bf16, size_t elem, float4 w) {
-  if (bf16) {
-    uint2 v;
-    v.x = pack_bf16x2_rn(w.x, w.y);
-    v.y = pack_bf16x2_rn(w.z, w.w);
-    *reinterpret_cast<uint2*>(static_cast<uint16_t*>(table) + elem) = v;
-  } else {
-    *reinterpret_cast<float4*>(static_cast<float*>(table) + elem) = w;
-  }
-}
-
-__device__ __forceinline__ float adagrad1(float& acc, float g, float w, const OptParams& p) {
-  acc = fmaf(g, g, acc);
-  return w - p.lr * g / (sqrtf(acc) + p.eps);
-}
-
-__device__ __forceinline__ float adam1(float& m, float& v, float g, float w, const OptParams& p) {
-  m = fmaf(p.beta1, m, p.omb1 * g);
-  v = fmaf(p.beta2, v, p.omb2 * g * g);
-  return w - p.lr * (m / p.bc1) / (sqrtf(v / p.bc2) + p.eps);
-}
 
 // Rows a lane group has in flight.  Measured on B200: Adam (four 16-byte streams per row) gains
 // from two rows a stride apart; Adagrad is faster with one row and the higher occupancy.
@@ -235,12 +198,7 @@ extern "C" int32_t antdt_sparse_opt_update(void* table, int32_t dtype, int64_t n
   if (!aligned16(table) || !aligned16(grads) || !aligned16(state1)) return ANTDT_ERR_INVALID_ARG;
   if (opt == ANTDT_OPT_ROWWISE_ADAGRAD ? (reinterpret_cast<uintptr_t>(state0) & 3u) != 0 : !aligned16(state0))
     return ANTDT_ERR_INVALID_ARG;
-  OptParams p;
-  p.lr = lr; p.eps = eps; p.beta1 = beta1; p.beta2 = beta2;
-  p.omb1 = (float)(1.0 - (double)beta1);
-  p.omb2 = (float)(1.0 - (double)beta2);
-  p.bc1 = (float)(1.0 - pow((double)beta1, (double)step));
-  p.bc2 = (float)(1.0 - pow((double)beta2, (double)step));
+  const OptParams p = make_opt_params(lr, eps, beta1, beta2, step);
   const bool adam = opt == ANTDT_OPT_ADAM, bf16 = dtype == ANTDT_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   const int nvec = dim / 4;
@@ -285,12 +243,7 @@ extern "C" int32_t antdt_dense_opt_update(float* params, const float* grad, int6
   if (!params || !grad || !state0 || (opt == ANTDT_OPT_ADAM && !state1)) return ANTDT_ERR_INVALID_ARG;
   if (!aligned16(params) || !aligned16(grad) || !aligned16(state0) || !aligned16(state1))
     return ANTDT_ERR_INVALID_ARG;
-  OptParams p;
-  p.lr = lr; p.eps = eps; p.beta1 = beta1; p.beta2 = beta2;
-  p.omb1 = (float)(1.0 - (double)beta1);
-  p.omb2 = (float)(1.0 - (double)beta2);
-  p.bc1 = (float)(1.0 - pow((double)beta1, (double)step));
-  p.bc2 = (float)(1.0 - pow((double)beta2, (double)step));
+  const OptParams p = make_opt_params(lr, eps, beta1, beta2, step);
   const int64_t n4 = n / 4;
   const int64_t want = (n4 + kOptThreads - 1) / kOptThreads;
   const int64_t cap = (int64_t)kNumSM * 16;

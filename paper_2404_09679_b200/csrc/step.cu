@@ -8,6 +8,25 @@
 #include "common.cuh"
 #include "segsort.cuh"
 
+namespace antdt {
+// The server half of a step: aggregate, then update; in one pass when the descriptor asks for it.
+static int32_t server_step(const antdt_step_desc* d, antdt_sparse_part* sp, const antdt_dense_part* dp,
+                           void* stream) {
+  if (d->fuse_update && (d->opt == ANTDT_OPT_ADAGRAD || d->opt == ANTDT_OPT_ADAM)) {
+    if (d->n_workers <= kRangeMaxWorkers) sp->agg_grads = nullptr;  // not materialised
+    return antdt_aggregate_update(sp, dp, d->batch_sizes, d->n_workers, d->table, d->dtype, d->opt,
+                                  d->lr, d->eps, d->beta1, d->beta2, d->step, d->state0, d->state1,
+                                  d->ws, d->ws_bytes, d->d_status, stream);
+  }
+  int32_t rc = antdt_weighted_aggregate(sp, dp, d->batch_sizes, d->n_workers, d->ws, d->ws_bytes,
+                                        d->d_status, stream);
+  if (rc != ANTDT_OK) return rc;
+  return antdt_sparse_opt_update(d->table, d->dtype, d->n_rows, d->dim, d->d_agg_ids, d->d_agg_grads,
+                                 d->d_n_agg, d->agg_cap, d->opt, d->lr, d->eps, d->beta1, d->beta2,
+                                 d->step, d->state0, d->state1, d->d_status, stream);
+}
+}  // namespace antdt
+
 namespace {
 // Side streams and events of the host-buffer step, created on first use for each device.
 constexpr int kMaxPieces = 16;  // the d_pooled copy is cut into at most this many pieces
@@ -138,12 +157,7 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
   sp.n_agg = d->d_n_agg; sp.out_cap = d->agg_cap;
   antdt_dense_part dp;
   dp.grads = d->d_dense_grads; dp.n = d->dense_n; dp.stride = d->dense_n; dp.out = d->d_dense_out;
-  rc = antdt_weighted_aggregate(&sp, dense ? &dp : nullptr, d->batch_sizes, d->n_workers, d->ws,
-                                d->ws_bytes, d->d_status, stream);
-  if (rc != ANTDT_OK) return rc;
-  rc = antdt_sparse_opt_update(d->table, d->dtype, d->n_rows, d->dim, d->d_agg_ids, d->d_agg_grads,
-                               d->d_n_agg, d->agg_cap, d->opt, d->lr, d->eps, d->beta1, d->beta2,
-                               d->step, d->state0, d->state1, d->d_status, stream);
+  rc = antdt::server_step(d, &sp, dense ? &dp : nullptr, stream);
   if (rc != ANTDT_OK) return rc;
   CK(cudaEventRecord(ss->done, s));
 
@@ -183,12 +197,7 @@ extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream)
   sp.n_agg = d->d_n_agg; sp.out_cap = d->agg_cap;
   antdt_dense_part dp;
   dp.grads = d->d_dense_grads; dp.n = d->dense_n; dp.stride = d->dense_n; dp.out = d->d_dense_out;
-  rc = antdt_weighted_aggregate(&sp, dense ? &dp : nullptr, d->batch_sizes, d->n_workers, d->ws,
-                                d->ws_bytes, d->d_status, stream);
-  if (rc != ANTDT_OK) return rc;
-  return antdt_sparse_opt_update(d->table, d->dtype, d->n_rows, d->dim, d->d_agg_ids, d->d_agg_grads,
-                                 d->d_n_agg, d->agg_cap, d->opt, d->lr, d->eps, d->beta1, d->beta2,
-                                 d->step, d->state0, d->state1, d->d_status, stream);
+  return antdt::server_step(d, &sp, dense ? &dp : nullptr, stream);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -233,7 +242,7 @@ std::vector<uint64_t> graph_key(const antdt_step_desc* d) {
       bits_of(d->d_uniq_ids), bits_of(d->d_worker_uniq_offsets), bits_of(d->d_seg_offsets),
       bits_of(d->d_sorted_occ), bits_of(d->d_uniq_grads), (uint64_t)d->uniq_cap,
       bits_of(d->d_agg_ids), bits_of(d->d_agg_grads), bits_of(d->d_n_agg), (uint64_t)d->agg_cap,
-      bits_of(d->ws), (uint64_t)d->ws_bytes, bits_of(d->d_status)};
+      bits_of(d->ws), (uint64_t)d->ws_bytes, bits_of(d->d_status), (uint64_t)(d->fuse_update != 0)};
   k.assign(head, head + sizeof(head) / sizeof(head[0]));
   for (int i = 0; i <= K; ++i) k.push_back((uint64_t)d->worker_sample_offsets[i]);
   for (int i = 0; i < K; ++i) k.push_back((uint64_t)d->batch_sizes[i]);

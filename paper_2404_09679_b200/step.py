@@ -73,10 +73,12 @@ class DeviceStep:
     """One antdt_bsp_step_device call per step: the descriptor is filled once for a buffer set and
     a model state, only the batch pointers and the step number change."""
 
-    def __init__(self, buf: StepBuffers, table, state0, state1, oc: OptConfig, n_workers: int):
+    def __init__(self, buf: StepBuffers, table, state0, state1, oc: OptConfig, n_workers: int,
+                 fuse_update: bool = False):
         import ctypes as C
         self.buf, self.K = buf, n_workers
         d = B.StepDesc()
+        d.fuse_update = 1 if fuse_update else 0
         p = lambda t: None if t is None else t.data_ptr()  # noqa: E731
         d.table, d.dtype = p(table), (B.BF16 if table.dtype == torch.bfloat16 else B.F32)
         d.n_rows, d.dim = table.shape
@@ -143,9 +145,10 @@ class HostStep:
     """antdt_bsp_step_host for a model state and a buffer set; `run` fills the descriptor for one
     batch given as page-locked host tensors and one HostStaging set."""
 
-    def __init__(self, buf: StepBuffers, table, state0, state1, oc: OptConfig, n_workers: int):
+    def __init__(self, buf: StepBuffers, table, state0, state1, oc: OptConfig, n_workers: int,
+                 fuse_update: bool = False):
         import ctypes as C
-        self._inner = DeviceStep(buf, table, state0, state1, oc, n_workers)
+        self._inner = DeviceStep(buf, table, state0, state1, oc, n_workers, fuse_update)
         self._C = C
 
     def run(self, st: HostStaging, step: int, h_row_ids, h_bag_offsets, bags_per_sample: int,
