@@ -55,6 +55,10 @@ int32_t bwd_dedup_impl(const int32_t* row_ids, int64_t nnz, const int64_t* bag_o
                        size_t ws_bytes, int32_t* dev_status, void* stream,
                        const PooledArrival* arrival);  // embbag_bwd.cu
 
+int32_t fwd_impl(const void* table, int32_t dtype, int64_t n_rows, int32_t dim, const int32_t* row_ids,
+                 int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,
+                 int32_t* dev_status, void* stream, int32_t bags_per_sample);  // embbag_fwd.cu
+
 constexpr int kNumSM = 148;  // B200: 2 dies x 74 SMs; grids are sized in multiples of this
 
 // ---- device helpers -------------------------------------------------------------------

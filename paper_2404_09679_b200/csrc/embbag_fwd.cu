@@ -13,17 +13,26 @@ namespace {
 constexpr int kFwdThreads = 128;
 constexpr int kFwdUnroll = 4;
 
-template <int G, int VPL, bool BF16>
-__global__ void __launch_bounds__(kFwdThreads)
+template <int G, int VPL, bool BF16, bool BY_FIELD>
+__global__ void __launch_bounds__(kFwdThreads, (VPL == 1 ? 12 : 1))
 embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
                   const int32_t* __restrict__ row_ids, int64_t nnz,
                   const int64_t* __restrict__ bag_offsets, int64_t n_bags,
-                  float* __restrict__ pooled, int32_t* status) {
+                  float* __restrict__ pooled, int32_t* status, int fields, int64_t sample_blocks) {
   constexpr int EPV = BF16 ? 8 : 4;   // elements per 16-byte vector
   constexpr int PAIRS = EPV / 2;      // packed fp32 pairs per vector
   constexpr int U = (G < kFwdUnroll) ? G : kFwdUnroll;
   const int lg = threadIdx.x & (G - 1);
-  const int64_t bag = (int64_t)blockIdx.x * (kFwdThreads / G) + (threadIdx.x / G);
+  // Bags are sample-major (bag = sample * fields + field).  When the caller knows `fields`, a CTA
+  // takes the bags of ONE field of consecutive samples and consecutive CTAs stay on that field,
+  // so that what is resident on an SM (and in L2) at one time draws from one field's hot rows.
+  int64_t bag;
+  if (BY_FIELD) {
+    const int64_t f = blockIdx.x / sample_blocks, sb = blockIdx.x % sample_blocks;
+    bag = (sb * (kFwdThreads / G) + (threadIdx.x / G)) * fields + f;
+  } else {
+    bag = (int64_t)blockIdx.x * (kFwdThreads / G) + (threadIdx.x / G);
+  }
   if (bag >= n_bags) return;
   const unsigned gmask = group_mask<G>();
   const int nvec = dim / EPV;
@@ -102,20 +111,30 @@ embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
 template <int G, int VPL, bool BF16>
 void launch_fwd(const void* table, int64_t n_rows, int dim, const int32_t* row_ids, int64_t nnz,
                 const int64_t* bag_offsets, int64_t n_bags, float* pooled, int32_t* status,
-                cudaStream_t s) {
+                cudaStream_t s, int fields) {
   const int64_t gpb = kFwdThreads / G;
-  const unsigned grid = (unsigned)((n_bags + gpb - 1) / gpb);
-  ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_kernel<G, VPL, BF16>), grid, kFwdThreads, 0, s, table,
-               n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status);
+  int64_t grid = (n_bags + gpb - 1) / gpb, sample_blocks = 0;
+  if (fields > 0 && n_bags % fields == 0) {
+    sample_blocks = (n_bags / fields + gpb - 1) / gpb;
+    grid = sample_blocks * fields;
+  } else {
+    fields = 0;
+  }
+  if (fields > 0)
+    ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_kernel<G, VPL, BF16, true>), (unsigned)grid, kFwdThreads, 0, s,
+                 table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status, fields, sample_blocks);
+  else
+    ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_kernel<G, VPL, BF16, false>), (unsigned)grid, kFwdThreads, 0, s,
+                 table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status, fields, sample_blocks);
 }
 
 template <bool BF16>
 int32_t dispatch_fwd(int nvec, const void* table, int64_t n_rows, int dim, const int32_t* row_ids,
                      int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,
-                     int32_t* status, cudaStream_t s) {
+                     int32_t* status, cudaStream_t s, int fields) {
 #define FWD_CASE(G, VPL)                                                                      \
   launch_fwd<G, VPL, BF16>(table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,     \
-                           status, s);                                                        \
+                           status, s, fields);                                                \
   return ANTDT_OK;
   if (nvec <= 1) { FWD_CASE(1, 1) }
   if (nvec <= 2) { FWD_CASE(2, 1) }
@@ -133,11 +152,11 @@ int32_t dispatch_fwd(int nvec, const void* table, int64_t n_rows, int dim, const
 }  // namespace
 }  // namespace antdt
 
-extern "C" int32_t antdt_embbag_fwd(const void* table, int32_t dtype, int64_t n_rows, int32_t dim,
-                                    const int32_t* row_ids, int64_t nnz,
-                                    const int64_t* bag_offsets, int64_t n_bags, float* pooled,
-                                    int32_t* dev_status, void* stream) {
-  using namespace antdt;
+namespace antdt {
+// The entry point's body; bags_per_sample > 0 (the step knows it) selects the field-major order.
+int32_t fwd_impl(const void* table, int32_t dtype, int64_t n_rows, int32_t dim, const int32_t* row_ids,
+                 int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,
+                 int32_t* dev_status, void* stream, int32_t bags_per_sample) {
   if (n_bags < 0 || nnz < 0 || n_rows < 1 || n_rows >= (1ll << 31) || nnz >= (1ll << 31) ||
       n_bags >= (1ll << 31) || dim < 1 || dim > 1024)
     return ANTDT_ERR_INVALID_ARG;
@@ -147,13 +166,26 @@ extern "C" int32_t antdt_embbag_fwd(const void* table, int32_t dtype, int64_t n_
   if (!table || !bag_offsets || !pooled || (nnz > 0 && !row_ids)) return ANTDT_ERR_INVALID_ARG;
   if (!aligned16(table) || !aligned16(pooled)) return ANTDT_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  // Field-major order pays when a bag's id list fills a 32-byte sector (eight ids or more on
+  // average): measured -12% on 100 fields x 10 ids x 256-byte rows, -2% on 40 x 20 x 128-byte rows,
+  // but +8% on 30 fields x 4.5 ids, where the scattered id reads cost more than the rows gain.
+  const int fields = (bags_per_sample > 1 && nnz >= 8 * n_bags) ? bags_per_sample : 0;
   int32_t rc;
   if (dtype == ANTDT_BF16)
     rc = dispatch_fwd<true>(dim / 8, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,
-                            dev_status, s);
+                            dev_status, s, fields);
   else
     rc = dispatch_fwd<false>(dim / 4, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags,
-                             pooled, dev_status, s);
+                             pooled, dev_status, s, fields);
   if (rc != ANTDT_OK) return rc;
   return cuda_ok();
+}
+}  // namespace antdt
+
+extern "C" int32_t antdt_embbag_fwd(const void* table, int32_t dtype, int64_t n_rows, int32_t dim,
+                                    const int32_t* row_ids, int64_t nnz,
+                                    const int64_t* bag_offsets, int64_t n_bags, float* pooled,
+                                    int32_t* dev_status, void* stream) {
+  return antdt::fwd_impl(table, dtype, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,
+                         dev_status, stream, 0);
 }

@@ -134,8 +134,9 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
   // compute on the caller's stream
   CK(cudaMemsetAsync(d->d_status, 0, 4, s));
   CK(cudaStreamWaitEvent(s, ss->ids, 0));
-  int32_t rc = antdt_embbag_fwd(d->table, d->dtype, d->n_rows, d->dim, d->d_row_ids, d->nnz,
-                                d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, stream);
+  int32_t rc = antdt::fwd_impl(d->table, d->dtype, d->n_rows, d->dim, d->d_row_ids, d->nnz,
+                               d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, stream,
+                               d->bags_per_sample);
   if (rc != ANTDT_OK) return rc;
   CK(cudaEventRecord(ss->fwd, s));
   CK(cudaStreamWaitEvent(ss->out, ss->fwd, 0));
@@ -181,8 +182,9 @@ extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream)
     return ANTDT_ERR_INVALID_ARG;
   const bool dense = d->d_dense_grads && d->dense_n > 0;
   if (dense && !d->d_dense_out) return ANTDT_ERR_INVALID_ARG;
-  int32_t rc = antdt_embbag_fwd(d->table, d->dtype, d->n_rows, d->dim, d->d_row_ids, d->nnz,
-                                d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, stream);
+  int32_t rc = antdt::fwd_impl(d->table, d->dtype, d->n_rows, d->dim, d->d_row_ids, d->nnz,
+                               d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, stream,
+                               d->bags_per_sample);
   if (rc != ANTDT_OK) return rc;
   rc = antdt_embbag_bwd_dedup(d->d_row_ids, d->nnz, d->d_bag_offsets, d->n_bags, d->bags_per_sample,
                               d->d_d_pooled, d->dim, d->n_rows, d->n_workers,

@@ -178,3 +178,30 @@ def test_two_host_steps_in_flight_equal_one_at_a_time():
     for (_, pa), (_, pb) in zip(o_a, o_b):
         assert torch.equal(pa, pb)
     assert torch.equal(t_a, t_b) and torch.equal(s_a, s_b)
+
+
+def test_device_step_forward_in_field_major_order_on_a_ragged_batch():
+    """The step knows the number of fields, so its forward walks the bags field by field (a CTA
+    takes one field of consecutive samples).  A sample count that fills neither the last CTA nor
+    the workers evenly, bags of 1..100 ids: pooled must equal the checker's and the bag-major
+    antdt_embbag_fwd's bit for bit."""
+    from paper_2404_09679_b200.step import DeviceStep
+    w = synth.WORKLOADS[4].scaled(B=1003, V=300_000)
+    plans = plan_steps(w, 1)
+    bm = synth.BatchMaker(w, "cuda")
+    table = bm.table()
+    batch = make_batch(bm, plans[0], 0)
+    nnz, n_bags = batch["row_ids"].numel(), batch["bag_offsets"].numel() - 1
+    assert n_bags == 1003 * w.F and nnz >= 8 * n_bags
+    oc = OptConfig(B.OPTS[w.opt], w.lr, w.eps, w.beta1, w.beta2)
+    buf = StepBuffers(w.D, w.K, nnz, n_bags, w.dense_n)
+    want = OracleState(w, table).step(batch, 1)["pooled"]
+    plain = torch.full((n_bags, w.D), float("nan"), device="cuda")
+    B.antdt_embbag_fwd(table, batch["row_ids"], batch["bag_offsets"], plain, buf.status)
+    ds = DeviceStep(buf, table.clone(), torch.zeros(w.V, w.D, device="cuda"), None, oc, w.K)
+    buf.pooled.fill_(float("nan"))
+    ds.run(1, batch["row_ids"], batch["bag_offsets"], w.F, batch["d_pooled"], batch["wso"].tolist(),
+           batch["counts"].tolist(), batch["dense"])
+    assert B.antdt_read_status(buf.status) == 0
+    assert torch.equal(buf.pooled[:n_bags], plain)
+    G.close(buf.pooled[:n_bags].cpu().numpy(), want)
