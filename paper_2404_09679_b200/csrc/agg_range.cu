@@ -23,12 +23,16 @@ constexpr int kRaBatch = 4;  // entries a thread loads before it processes them
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // ---------------------------------------------------------------------------------------
+struct WeightBlob { float w[kRangeMaxWorkers]; };  // the workers' weights, a kernel parameter
+
 __global__ void __launch_bounds__(kRaThreads)
 range_split_kernel(const int32_t* __restrict__ ids, const int64_t* __restrict__ wuo_in, int K,
                    int64_t in_cap, int r_log2, int64_t P, uint32_t dropped,
                    int64_t* __restrict__ wuo_out, int64_t* __restrict__ n_entries,
-                   int32_t* __restrict__ bnd, int32_t* status) {
+                   int32_t* __restrict__ bnd, const WeightBlob weights, float* __restrict__ weights_out,
+                   int32_t* status) {
   __shared__ int64_t s_wuo[kRangeMaxWorkers + 1];
+  if (blockIdx.x == 0 && weights_out && threadIdx.x < K) weights_out[threadIdx.x] = weights.w[threadIdx.x];
   if (threadIdx.x == 0) {  // ascending and inside [0, in_cap], whatever came in
     int64_t prev = 0, kept = 0;
     for (int i = 0; i <= K; ++i) {
@@ -362,9 +366,12 @@ void range_prepare_device() {
 void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t in_cap, int64_t n_rows,
                        int K, uint32_t dropped_bits, int32_t* agg_ids, int64_t* n_agg, int64_t out_cap,
                        int64_t* wuo_out, int64_t* n_entries, uint32_t* src, uint32_t* head_bits,
-                       int32_t* tile_first, int tile, uint32_t* row_start, char* ws, const RangeLayout& L,
-                       int32_t* status, cudaStream_t s) {
+                       int32_t* tile_first, int tile, uint32_t* row_start, const float* weights_host,
+                       float* weights_dev, char* ws, const RangeLayout& L, int32_t* status,
+                       cudaStream_t s) {
   range_prepare_device();
+  WeightBlob wb;
+  for (int i = 0; i < kRangeMaxWorkers; ++i) wb.w[i] = (weights_host && i < K) ? weights_host[i] : 0.f;
   const int r_log2 = range_log2(n_rows, in_cap);
   const int64_t P = (n_rows + ((int64_t)1 << r_log2) - 1) >> r_log2;  // <= kRangeMaxRanges
   int32_t* bnd = (int32_t*)(ws + L.bnd);
@@ -375,7 +382,7 @@ void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t i
   const int64_t n_search = (int64_t)K * (P + 1);
   ANTDT_LAUNCH("agg_range_split", range_split_kernel, (unsigned)((n_search + kRaThreads - 1) / kRaThreads),
                kRaThreads, 0, s, uniq_ids, wuo_in, K, in_cap, r_log2, P, dropped_bits, wuo_out, n_entries,
-               bnd, status);
+               bnd, wb, weights_host ? weights_dev : nullptr, status);
   ANTDT_LAUNCH("agg_range_count", range_count_kernel, (unsigned)P, kRaThreads, 0, s,
                uniq_ids, bnd, wuo_out, K, P, r_log2, n_rows, dropped_bits, distinct, status);
   ANTDT_LAUNCH("agg_range_scan", range_scan_kernel, 1, 1024, 0, s, distinct, P, base, n_agg, out_cap,

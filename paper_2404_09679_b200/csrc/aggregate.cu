@@ -400,7 +400,9 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
   float hw[kMaxSegments];
   for (int i = 0; i < K; ++i)
     hw[i] = (dropped && dropped[i]) ? 0.f : (float)((double)batch_sizes[i] / tot);
-  upload_small(hw, 4 * (size_t)K, w8 + L.weights, s);
+  // the range merge (up to 32 workers, sparse part present) carries the weights itself
+  const bool by_ranges = sp && K <= kRangeMaxWorkers && in_cap > 0;
+  if (!by_ranges) upload_small(hw, 4 * (size_t)K, w8 + L.weights, s);
 
   if (sp) {
     int64_t* bounds = (int64_t*)(w8 + L.bounds);
@@ -414,7 +416,8 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
                         sp->agg_ids, sp->n_agg, agg_cap, (int64_t*)(w8 + L.wuo), bounds,
                         (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.head_bits),
                         (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap),
-                        fu ? (uint32_t*)(w8 + L.row_start) : nullptr, w8 + L.range_ws, L.range, dev_status, s);
+                        fu ? (uint32_t*)(w8 + L.row_start) : nullptr, hw, (float*)(w8 + L.weights),
+                        w8 + L.range_ws, L.range, dev_status, s);
     } else {
       sort_merge_order(sp, dropped, any_dropped, K, in_cap, agg_cap, w8, L, dev_status, s);
     }
@@ -456,7 +459,7 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
       t.out = sp->agg_grads;
       t.head_part = (float*)(w8 + L.head_part);
       t.tail_part = (float*)(w8 + L.tail_part);
-      launch_tile_reduce<true>(t, "agg_reduce", "agg_fixup", s);
+      launch_tile_reduce(t, "agg_reduce", "agg_fixup", s);
     }
   }
   if (dp && dp->n > 0) {

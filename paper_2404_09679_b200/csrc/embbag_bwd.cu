@@ -161,10 +161,14 @@ int32_t bwd_dedup_impl(
   uint32_t* vals_t = (uint32_t*)(w8 + L.vals_t);
   char* sort_ws = w8 + L.sort_ws;
 
-  upload_small(worker_sample_offsets, 8 * ((size_t)K + 1), d_wso, s);
-  ANTDT_LAUNCH("bwd_prep", bwd_prep_kernel, 1, 1024, 0, s, d_wso, K, (int)bags_per_sample,
-               bag_offsets, n_bags, nnz, d_occ_bounds, d_worker_b, dev_status);
-  segsort_setup(d_occ_bounds, K, nnz, sort_ws, L.sort, s);
+  // one launch for up to 255 workers; beyond that the offsets travel in pieces
+  if (!segsort_setup_workers(worker_sample_offsets, K, (int)bags_per_sample, bag_offsets, n_bags, nnz,
+                             d_worker_b, sort_ws, L.sort, dev_status, s)) {
+    upload_small(worker_sample_offsets, 8 * ((size_t)K + 1), d_wso, s);
+    ANTDT_LAUNCH("bwd_prep", bwd_prep_kernel, 1, 1024, 0, s, d_wso, K, (int)bags_per_sample,
+                 bag_offsets, n_bags, nnz, d_occ_bounds, d_worker_b, dev_status);
+    segsort_setup(d_occ_bounds, K, nnz, sort_ws, L.sort, s);
+  }
 
   const int key_bits = bits_for(n_rows);
   const int P = sort_passes(key_bits);

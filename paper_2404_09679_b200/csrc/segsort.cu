@@ -46,10 +46,11 @@ __device__ int64_t block_exclusive_scan_1024(int64_t v, int64_t* total, int64_t*
 // ---------------------------------------------------------------------------------------
 // setup: sanitise the segment bounds and cut the segments into chunks
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-segsort_setup_kernel(const int64_t* __restrict__ bounds_in, int S, int64_t n_cap, SortDesc* desc,
-                     int64_t* seg_bounds, int32_t* seg_first, int32_t* chunk_seg,
-                     int64_t* chunk_begin, int64_t* chunk_end, int max_chunks) {
+// The body of the set-up, run by one CTA of 1024 threads.  bounds_in may be global or shared memory.
+__device__ __forceinline__ void segsort_setup_body(const int64_t* bounds_in, int S, int64_t n_cap,
+                                                   SortDesc* desc, int64_t* seg_bounds, int32_t* seg_first,
+                                                   int32_t* chunk_seg, int64_t* chunk_begin,
+                                                   int64_t* chunk_end, int max_chunks) {
   __shared__ int64_t sb[kMaxSegments + 1];
   __shared__ int32_t sf[kMaxSegments + 1];
   __shared__ int64_t s_chunk_elems;
@@ -100,6 +101,36 @@ segsort_setup_kernel(const int64_t* __restrict__ bounds_in, int S, int64_t n_cap
     chunk_begin[c] = b;
     chunk_end[c] = min(b + ce, sb[lo + 1]);
   }
+}
+
+__global__ void __launch_bounds__(1024)
+segsort_setup_kernel(const int64_t* __restrict__ bounds_in, int S, int64_t n_cap, SortDesc* desc,
+                     int64_t* seg_bounds, int32_t* seg_first, int32_t* chunk_seg,
+                     int64_t* chunk_begin, int64_t* chunk_end, int max_chunks) {
+  segsort_setup_body(bounds_in, S, n_cap, desc, seg_bounds, seg_first, chunk_seg, chunk_begin, chunk_end,
+                     max_chunks);
+}
+
+// The backward's set-up in one launch: the workers' sample offsets arrive as a kernel parameter,
+// their occurrence ranges are read off bag_offsets (the segments of the sort), 1/b_w is written,
+// the offsets' ends are checked, and the chunks are cut as above.
+struct WorkerBlob { int64_t wso[kSetupMaxWorkers + 1]; };
+__global__ void __launch_bounds__(1024)
+bwd_setup_kernel(const WorkerBlob blob, int K, int F, const int64_t* __restrict__ bag_offsets,
+                 int64_t n_bags, int64_t nnz, float* __restrict__ worker_b, SortDesc* desc,
+                 int64_t* seg_bounds, int32_t* seg_first, int32_t* chunk_seg, int64_t* chunk_begin,
+                 int64_t* chunk_end, int max_chunks, int32_t* status) {
+  __shared__ int64_t s_occ[kSetupMaxWorkers + 1];
+  const int tid = threadIdx.x;
+  if (tid == 0 && (bag_offsets[0] != 0 || bag_offsets[n_bags] != nnz))
+    set_status(status, ANTDT_ERR_BAD_OFFSETS);
+  for (int w = tid; w <= K; w += blockDim.x) {
+    s_occ[w] = bag_offsets[blob.wso[w] * (int64_t)F];  // host checked: 0 <= bag <= n_bags
+    if (w < K) worker_b[w] = 1.0f / (float)(blob.wso[w + 1] - blob.wso[w]);  // inf for an empty worker: unused
+  }
+  __syncthreads();
+  segsort_setup_body(s_occ, K, nnz, desc, seg_bounds, seg_first, chunk_seg, chunk_begin, chunk_end,
+                     max_chunks);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -572,6 +603,20 @@ void segsort_setup(const int64_t* seg_bounds_dev, int S, int64_t n_cap, char* ws
                (SortDesc*)(ws + L.desc), (int64_t*)(ws + L.seg_bounds),
                (int32_t*)(ws + L.seg_first), (int32_t*)(ws + L.chunk_seg),
                (int64_t*)(ws + L.chunk_begin), (int64_t*)(ws + L.chunk_end), L.max_chunks);
+}
+
+bool segsort_setup_workers(const int64_t* wso_host, int K, int F, const int64_t* bag_offsets,
+                           int64_t n_bags, int64_t nnz, float* worker_b, char* ws, const SortLayout& L,
+                           int32_t* status, cudaStream_t s) {
+  if (K > kSetupMaxWorkers) return false;
+  WorkerBlob blob;
+  for (int i = 0; i <= K; ++i) blob.wso[i] = wso_host[i];
+  for (int i = K + 1; i <= kSetupMaxWorkers; ++i) blob.wso[i] = 0;
+  ANTDT_LAUNCH("bwd_setup", bwd_setup_kernel, 1, 1024, 0, s, blob, K, F, bag_offsets, n_bags, nnz, worker_b,
+               (SortDesc*)(ws + L.desc), (int64_t*)(ws + L.seg_bounds), (int32_t*)(ws + L.seg_first),
+               (int32_t*)(ws + L.chunk_seg), (int64_t*)(ws + L.chunk_begin), (int64_t*)(ws + L.chunk_end),
+               L.max_chunks, status);
+  return true;
 }
 
 // Per device, once: opt in to the scatter's 55 KB of dynamic shared memory (3 CTAs per SM).

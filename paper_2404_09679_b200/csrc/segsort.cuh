@@ -24,6 +24,7 @@ constexpr int kSortTile = kSortThreads * kSortItems;  // 4096 pairs staged in sh
 constexpr int kSortMaxBits = 9;                       // up to 512 bins per pass
 constexpr int kSortMaxBins = 1 << kSortMaxBits;
 constexpr int kMaxSegments = 1024;
+constexpr int kSetupMaxWorkers = 255;  // worker offsets that fit one kernel-parameter blob (2 KB)
 
 // Device-side description of the chunks (written by segsort_setup, read by every pass).
 struct SortDesc {
@@ -67,6 +68,14 @@ void segsort_prepare_device();
 // chunk descriptors in `ws` (laid out by sort_layout).
 void segsort_setup(const int64_t* seg_bounds_dev, int n_segments, int64_t n_cap, char* ws,
                    const SortLayout& L, cudaStream_t s);
+
+// The backward's set-up in ONE launch when there are at most kSetupMaxWorkers workers: takes the
+// host's worker_sample_offsets [K+1] as a kernel parameter, derives every worker's occurrence
+// range from bag_offsets (these are the sort's segments), writes 1/b_w to worker_b [K], checks the
+// ends of bag_offsets, and builds the chunk descriptors.  false: too many workers, nothing launched.
+bool segsort_setup_workers(const int64_t* wso_host, int n_workers, int bags_per_sample,
+                           const int64_t* bag_offsets, int64_t n_bags, int64_t nnz, float* worker_b,
+                           char* ws, const SortLayout& L, int32_t* status, cudaStream_t s);
 
 // Sorts by the low key_bits bits.  keys_in is read only; the sorted pairs land in
 // keys_out/vals_out; keys_tmp/vals_tmp are scratch of the same size.  vals_in == nullptr means

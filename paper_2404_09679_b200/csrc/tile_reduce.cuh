@@ -1,23 +1,19 @@
-// Tile-parallel segmented reduction of gathered rows, shared by the worker backward (sum of
-// d_pooled rows per (worker, row) run, scaled by 1/b_w) and the server aggregation (weighted sum
-// of the workers' gradient rows per row).
+// Tile-parallel segmented reduction of gathered rows for the server aggregation: the weighted sum
+// of the workers' gradient rows per aggregated row.  (The worker backward has its own walk,
+// bwd_walk.cuh, built on the same tiles.)
 //
-// The sorted array of payloads (row indices into `rows`) is cut into tiles of 64 (16 for a small
-// input) consecutive entries whatever runs they belong to, so the work is balanced by entries, not by
-// runs: a run holding 20% of a field costs its tiles no more than anyone else's.  A group of G
-// lanes (one 16-byte vector of the row per lane and VPL step) walks one tile; a run that starts
-// and ends inside the tile is written out, the pieces of runs that cross the tile's edges go to
-// head_part / tail_part, and the fix-up pass lets the tile where such a run STARTS add its tail
-// piece and the following head pieces in tile order.  Every sum has a fixed order: no
-// floating-point atomics, bit-reproducible.
+// The merge-order array of payloads (row indices into `rows`) is cut into tiles of 64 (16 for a
+// small input) consecutive entries whatever runs they belong to, so the work is balanced by
+// entries, not by runs.  A group of G lanes (one 16-byte vector of the row per lane and VPL step)
+// walks one tile; a run that starts and ends inside the tile is written out, the pieces of runs
+// that cross the tile's edges go to head_part / tail_part, and the fix-up pass lets the tile where
+// such a run STARTS add its tail piece and the following head pieces in tile order.  Every sum has
+// a fixed order (ascending worker inside a row): no floating-point atomics, bit-reproducible.
 //
-// The walk is issue-bound once the gathered rows sit in L1/L2, so it is built to cost few
-// instructions per entry: the tile's run ends are one 64-bit mask consumed with constant
-// shifts and tested once per kRedUnroll entries (inside a hot row nothing closes, and the
-// entries are only added), the payloads of G entries live in one register per lane and are
-// broadcast by shuffle, kRedUnroll row loads are in flight before the first add, the backward's
-// loads are unconditional (clamped indices instead of predicates), and the worker (for the 1/b_w
-// scale) is only re-resolved when the walk crosses a worker boundary.
+// The payloads of G entries live in one register per lane and are broadcast by shuffle,
+// kRedUnroll row loads are in flight before the first add, slots without data are predicated off,
+// and every entry carries its worker's weight (found by a search of the position in the workers'
+// offsets, done once per lane and broadcast).
 #pragma once
 #include "common.cuh"
 
@@ -42,13 +38,13 @@ struct TileArgs {
   int64_t n_host;             // entries (upper bound when n_dev is given)
   const int64_t* n_dev;       // device-side entry count or nullptr
   int64_t payload_limit;      // rows of the matrix (>= 1); a payload >= this reads the last row
-  const int64_t* bounds;      // backward: entry range of every worker [K+1];
+  const int64_t* bounds;      // backward walk: entry range of every worker [K+1];
                               // aggregation: payload range of every worker [K+1]
-  const float* scales;        // backward: 1/b_w [K]; aggregation: weight w_i [K]
+  const float* scales;        // backward walk: 1/b_w [K]; aggregation: weight w_i [K]
   int K;
   int64_t out_cap;
   float* out;                 // [out_cap, dim]
-  float* head_part;           // [n_tiles, dim]
+  float* head_part;           // [n_tiles, dim]   (aggregation; the backward walk has its own scratch)
   float* tail_part;           // [n_tiles, dim]
   // Which part of the work a launch_tile_reduce call issues (defaults: everything).  A caller
   // whose `rows` arrive in pieces walks the tiles piece by piece and runs the fix-up last.
@@ -60,18 +56,17 @@ struct TileArgs {
 
 // The hot pointers are separate __restrict__ parameters (not read through the struct) so that
 // the compiler may move row loads across the run-end stores.
-template <int G, int VPL, bool AGG, int TILE>
+template <int G, int VPL, int TILE>
 __global__ void __launch_bounds__(kRedThreads, (VPL == 1 ? 6 : 1))
 tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
                    const uint32_t* __restrict__ head_bits, const int32_t* __restrict__ tile_first,
                    const float* __restrict__ rows, float* __restrict__ out,
                    float* __restrict__ head_part, float* __restrict__ tail_part) {
-  extern __shared__ int64_t s_bounds[];  // [K+1], then K floats (aggregation)
+  extern __shared__ int64_t s_bounds[];  // payload range of every worker [K+1], then K weights
   float* s_w = reinterpret_cast<float*>(s_bounds + (a.K + 1));
   const int K = a.K;
   for (int i = threadIdx.x; i <= K; i += blockDim.x) s_bounds[i] = a.bounds[i];
-  if (AGG)
-    for (int i = threadIdx.x; i < K; i += blockDim.x) s_w[i] = a.scales[i];
+  for (int i = threadIdx.x; i < K; i += blockDim.x) s_w[i] = a.scales[i];
   __syncthreads();
   const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
   const int lg = threadIdx.x & (G - 1);
@@ -97,53 +92,29 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
     started = (h0 & 1u) != 0;
   } else {  // TILE < 32 and a power of two: the tile's bits and the next one lie in two words
     const uint64_t heads = ((uint64_t)__ldg(hw) | ((uint64_t)__ldg(hw + 1) << 32)) >> (o_begin & 31);
-    ends = (heads >> 1) & ((1ull << TILE) - 1ull);
-    open_tail = !last_tile && !((heads >> TILE) & 1ull);
+    ends = (heads >> 1) & ((1ull << (TILE & 63)) - 1ull);
+    open_tail = !last_tile && !((heads >> (TILE & 63)) & 1ull);
     started = (heads & 1ull) != 0;
   }
   if (last_tile) ends = (ends & ((1ull << (nv - 1)) - 1ull)) | (1ull << (nv - 1));  // array end closes
 
   int64_t u = tile_first[tile];
-  int w = 0, next_w_rel = TILE + 1;
-  float inv = 1.f;
-  if (!AGG) {
-    w = interval_of(s_bounds, K + 1, o_begin);
-    if (w > K - 1) w = K - 1;
-    // tile-relative position at which the next worker starts (beyond the tile: never reached)
-    next_w_rel = (int)min((int64_t)(TILE + 1), s_bounds[w + 1] - o_begin);
-    inv = a.scales[w];
-  }
-
   float4 acc[VPL];
 #pragma unroll
   for (int k = 0; k < VPL; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
   const uint32_t row_stride = (uint32_t)dim;
 
-  // Every load of the backward's walk is unconditional: a payload outside the matrix (only possible after
-  // an error that is already flagged) is clamped to the last row, idle lanes of a row whose width
-  // is not a power of two re-read its last vector, and the slots past the data of the last tile
-  // read row 0 - they come after the bit that closes the last run, so their sum is never stored.
   constexpr int GE = G < TILE ? G : TILE;  // entries a group step covers
-  const uint32_t last_row = (uint32_t)(a.payload_limit - 1);
-  int vi_c[VPL];
-#pragma unroll
-  for (int k = 0; k < VPL; ++k) vi_c[k] = min(lg + k * G, nvec - 1);
   for (int q = 0; q * GE < nv; ++q) {
-    // backward: unconditional loads as described above.  Aggregation (bound by DRAM, and its
-    // weight lookup already fills the register budget): slots without data are marked -1 and
-    // their loads predicated off.
-    int my_row = AGG ? -1 : 0;
+    // slots without data are marked -1 and their loads predicated off
+    int my_row = -1;
     float my_wt = 0.f;
     if (lg < GE && q * GE + lg < nv) {
       const uint32_t p = __ldg(payload + o_begin + q * GE + lg);
-      if (AGG) {
-        my_row = ((int64_t)p < a.payload_limit) ? (int)p : -1;
-        if (my_row >= 0) {
-          int wl = interval_of(s_bounds, K + 1, (int64_t)p);
-          my_wt = s_w[wl > K - 1 ? K - 1 : wl];
-        }
-      } else {
-        my_row = (int)min(p, last_row);
+      my_row = ((int64_t)p < a.payload_limit) ? (int)p : -1;
+      if (my_row >= 0) {
+        int wl = interval_of(s_bounds, K + 1, (int64_t)p);
+        my_wt = s_w[wl > K - 1 ? K - 1 : wl];
       }
     }
 #pragma unroll
@@ -153,71 +124,30 @@ tile_reduce_kernel(const TileArgs a, const uint32_t* __restrict__ payload,
 #pragma unroll
       for (int t = 0; t < U; ++t) {
         const int row = __shfl_sync(gmask, my_row, j0 + t, G);
-        wt[t] = AGG ? __shfl_sync(gmask, my_wt, j0 + t, G) : 1.f;
-        if (AGG) {
-          const float* rp = rows + (size_t)((uint32_t)(row < 0 ? 0 : row)) * row_stride;
+        wt[t] = __shfl_sync(gmask, my_wt, j0 + t, G);
+        const float* rp = rows + (size_t)((uint32_t)(row < 0 ? 0 : row)) * row_stride;
 #pragma unroll
-          for (int k = 0; k < VPL; ++k) {
-            const int vi = lg + k * G;
-            v[t][k] = (row >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-        } else {
-          const float* rp = rows + (size_t)(uint32_t)row * row_stride;
-#pragma unroll
-          for (int k = 0; k < VPL; ++k) v[t][k] = ldg_f4(rp + 4 * vi_c[k]);
+        for (int k = 0; k < VPL; ++k) {
+          const int vi = lg + k * G;
+          v[t][k] = (row >= 0 && vi < nvec) ? ldg_f4(rp + 4 * vi) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-      }
-      if (!AGG && ((ends >> j0) & ((1ull << U) - 1ull)) == 0ull) {
-        // none of these U entries closes a run (the common case inside a hot row): add, no tests
-#pragma unroll
-        for (int t = 0; t < U; ++t) {
-#pragma unroll
-          for (int k = 0; k < VPL; ++k) {
-            acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
-            acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
-          }
-        }
-        continue;
       }
 #pragma unroll
       for (int t = 0; t < U; ++t) {
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-          if (AGG) {
-            acc[k].x = fmaf(wt[t], v[t][k].x, acc[k].x); acc[k].y = fmaf(wt[t], v[t][k].y, acc[k].y);
-            acc[k].z = fmaf(wt[t], v[t][k].z, acc[k].z); acc[k].w = fmaf(wt[t], v[t][k].w, acc[k].w);
-          } else {
-            acc[k].x += v[t][k].x; acc[k].y += v[t][k].y;
-            acc[k].z += v[t][k].z; acc[k].w += v[t][k].w;
-          }
+          acc[k].x = fmaf(wt[t], v[t][k].x, acc[k].x); acc[k].y = fmaf(wt[t], v[t][k].y, acc[k].y);
+          acc[k].z = fmaf(wt[t], v[t][k].z, acc[k].z); acc[k].w = fmaf(wt[t], v[t][k].w, acc[k].w);
         }
         if ((ends >> (j0 + t)) & 1ull) {  // this entry closes its run
           float* dst;
-          float sc = 1.f;
-          if (started) {
-            if (!AGG) {
-              const int rel = q * GE + j0 + t;
-              if (rel >= next_w_rel) {  // crossed into a later worker's range
-                const int64_t o = o_begin + rel;
-                while (w < K - 1 && o >= s_bounds[w + 1]) ++w;
-                next_w_rel = (int)min((int64_t)(TILE + 1), s_bounds[w + 1] - o_begin);
-                if (w == K - 1) next_w_rel = TILE + 1;
-                inv = a.scales[w];
-              }
-              sc = inv;
-            }
-            dst = (u < a.out_cap) ? out + (size_t)u * row_stride : nullptr;
-          } else {
-            dst = head_part + (size_t)tile * row_stride;
-          }
+          if (started) dst = (u < a.out_cap) ? out + (size_t)u * row_stride : nullptr;
+          else dst = head_part + (size_t)tile * row_stride;
           if (dst) {
 #pragma unroll
             for (int k = 0; k < VPL; ++k) {
               const int vi = lg + k * G;
-              if (vi < nvec)
-                reinterpret_cast<float4*>(dst)[vi] =
-                    AGG ? acc[k]
-                        : make_float4(acc[k].x * sc, acc[k].y * sc, acc[k].z * sc, acc[k].w * sc);
+              if (vi < nvec) reinterpret_cast<float4*>(dst)[vi] = acc[k];
             }
           }
           ++u;
@@ -254,7 +184,7 @@ __device__ __forceinline__ bool head_at(const uint32_t* __restrict__ hb, int64_t
 
 // Fix-up: the tile in which a straddling run STARTS owns it.  total = its tail piece, then
 // the head pieces of the following tiles in order until the run ends.
-template <int G, int VPL, bool AGG, int TILE>
+template <int G, int VPL, int TILE>
 __global__ void __launch_bounds__(kRedThreads)
 tile_fixup_kernel(const TileArgs a) {
   const int64_t n = a.n_dev ? min(*a.n_dev, a.n_host) : a.n_host;
@@ -283,12 +213,6 @@ tile_fixup_kernel(const TileArgs a) {
                 : make_float4(0.f, 0.f, 0.f, 0.f);
     nxt[k] = in ? reinterpret_cast<const float4*>(a.head_part + (size_t)(tile + 1) * dim)[vi]
                 : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  float scale = 1.f;
-  if (!AGG) {  // worker of the run = worker of any of its entries (searched while the loads fly)
-    int w = interval_of(a.bounds, a.K + 1, o_end - 1);
-    if (w > a.K - 1) w = a.K - 1;
-    scale = a.scales[w];
   }
   if (nxt_heads & 1ull) return;  // next tile starts a new run: nothing straddles
   const int heads = __popcll(cur);
@@ -319,14 +243,11 @@ tile_fixup_kernel(const TileArgs a) {
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
     const int vi = lg + k * G;
-    if (vi >= nvec) continue;
-    float4 r = tot[k];
-    if (!AGG) { r.x *= scale; r.y *= scale; r.z *= scale; r.w *= scale; }
-    reinterpret_cast<float4*>(dst)[vi] = r;
+    if (vi < nvec) reinterpret_cast<float4*>(dst)[vi] = tot[k];
   }
 }
 
-template <int G, int VPL, bool AGG, int TILE>
+template <int G, int VPL, int TILE>
 void launch_tile_reduce_t(const TileArgs& a_in, const char* name_tiles, const char* name_fixup,
                           cudaStream_t s) {
   const int64_t n_tiles = (a_in.n_host + TILE - 1) / TILE;
@@ -334,30 +255,29 @@ void launch_tile_reduce_t(const TileArgs& a_in, const char* name_tiles, const ch
   TileArgs a = a_in;
   if (a.tile_begin < 0) a.tile_begin = 0;
   if (a.tile_end < 0 || a.tile_end > n_tiles) a.tile_end = n_tiles;
-  const size_t smem = 8 * ((size_t)a.K + 1) + (AGG ? 4 * (size_t)a.K : 0);
+  const size_t smem = 8 * ((size_t)a.K + 1) + 4 * (size_t)a.K;
   if (a.walk && a.tile_end > a.tile_begin) {
     const unsigned grid = (unsigned)((a.tile_end - a.tile_begin + tpb - 1) / tpb);
-    ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, smem, s, a,
+    ANTDT_LAUNCH(name_tiles, (tile_reduce_kernel<G, VPL, TILE>), grid, kRedThreads, smem, s, a,
                  a.payload, a.head_bits, a.tile_first, a.rows, a.out, a.head_part, a.tail_part);
   }
   if (a.fixup && n_tiles > 0) {
     const unsigned grid = (unsigned)((n_tiles + tpb - 1) / tpb);
-    ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, AGG, TILE>), grid, kRedThreads, 0, s, a);
+    ANTDT_LAUNCH(name_fixup, (tile_fixup_kernel<G, VPL, TILE>), grid, kRedThreads, 0, s, a);
   }
 }
 
-template <int G, int VPL, bool AGG>
+template <int G, int VPL>
 void launch_tile_reduce_gv(const TileArgs& a, const char* name_tiles, const char* name_fixup,
                            cudaStream_t s) {
-  if (a.tile == kRedTileSmall) launch_tile_reduce_t<G, VPL, AGG, kRedTileSmall>(a, name_tiles, name_fixup, s);
-  else launch_tile_reduce_t<G, VPL, AGG, kRedTile>(a, name_tiles, name_fixup, s);
+  if (a.tile == kRedTileSmall) launch_tile_reduce_t<G, VPL, kRedTileSmall>(a, name_tiles, name_fixup, s);
+  else launch_tile_reduce_t<G, VPL, kRedTile>(a, name_tiles, name_fixup, s);
 }
 
-template <bool AGG>
-void launch_tile_reduce(const TileArgs& a, const char* name_tiles, const char* name_fixup,
-                        cudaStream_t s) {
+inline void launch_tile_reduce(const TileArgs& a, const char* name_tiles, const char* name_fixup,
+                               cudaStream_t s) {
   const int nvec = a.dim / 4;
-#define TILE_CASE(G, VPL) launch_tile_reduce_gv<G, VPL, AGG>(a, name_tiles, name_fixup, s)
+#define TILE_CASE(G, VPL) launch_tile_reduce_gv<G, VPL>(a, name_tiles, name_fixup, s)
   if (nvec <= 1) TILE_CASE(1, 1);
   else if (nvec <= 2) TILE_CASE(2, 1);
   else if (nvec <= 4) TILE_CASE(4, 1);
