@@ -45,3 +45,25 @@ def test_reference_arm_prints_its_line():
     assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0,
                         "d2h_bytes_per_step": 0}
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
+
+
+def test_roofline_fraction_is_a_dram_fraction_and_the_l2_roof_is_reported():
+    d = _run("--config", "2", "--steps", "3", "--warmup", "3", "--no-cpu-baseline", "--no-e2e")
+    r = d["roofline"]
+    assert r["frac"] is None or 0 < r["frac"] < 1.3        # what DRAM did, never a cache-served rate
+    assert "frac_source" in r and "frac_algorithmic" in r
+    g = d["l2_gather"]
+    assert g and all(v["l2_gather_peak_GBps"] > 1000 and 0 < v["frac_of_l2_gather_peak"] < 1.5 for v in g.values())
+
+
+@pytest.mark.parametrize("case", ["dense_adagrad", "dense_adam", "rowwise_adagrad", "rowwise_adagrad_bf16",
+                                  "aggregate_k33", "aggregate_backup", "fused_adagrad_bf16", "fused_adam"])
+def test_kernel_bench_cases_run(case, monkeypatch, capsys):
+    if ROOT not in sys.path:
+        sys.path.insert(0, ROOT)
+    from paper_2404_09679_b200 import kernel_bench
+    monkeypatch.setattr(sys, "argv", ["kernel_bench", "--case", case, "--n", "65536", "--rows", "20000",
+                                      "--table-rows", "100000", "--dim", "32", "--reps", "2"])
+    kernel_bench.main()
+    d = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
+    assert d["case"] == case and d["ms_per_call"] > 0 and d["kernels_ms_per_launch"]
