@@ -440,8 +440,20 @@ int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream);
  *     executables are driver objects, the only thing this library ever creates on a device.
  *   - Per-kernel event timing (antdt_profile_enable) does not see kernels inside a graph;
  *     antdt_launch_count counts a replay's kernel nodes.
+ *   - Small batches (at most 2^22 occurrences, at most 32 workers, no fuse_update) are captured
+ *     as three branches when the workspace has room: the forward beside the backward, and the
+ *     aggregation's merge order (which needs the workers' id lists, not their gradients) beside
+ *     the backward's sums.  No kernel fills the device there, so the step time is the length of
+ *     the dependency chain.  The results are those of the one-chain step.  Room means ws_bytes
+ *     >= antdt_bsp_step_workspace_bytes(...): the aggregation's scratch then sits behind the
+ *     backward's instead of on top of it.  The branches use two library-owned side streams.
  * Returns ANTDT_OK, an argument error, or ANTDT_ERR_CUDA. */
 int32_t antdt_bsp_step_graph(const antdt_step_desc* d, void* stream);
+/* Workspace of a step: the larger of the backward's and the aggregation's figures; their sum
+ * (the backward's rounded up to 256 bytes) for a batch small enough for the three-branch graph.
+ * 0 for arguments either figure rejects. */
+size_t antdt_bsp_step_workspace_bytes(int64_t nnz, int64_t n_bags, int32_t dim, int32_t n_workers,
+                                      int64_t uniq_cap);
 /* Destroys the executable graphs kept for the current device. */
 int32_t antdt_bsp_step_graph_reset(void);
 

@@ -33,6 +33,7 @@ EXPORTS = [
     "antdt_embbag_bwd_dedup",
     "antdt_embbag_bwd_dedup_static",
     "antdt_weighted_aggregate_workspace_bytes", "antdt_weighted_aggregate",
+    "antdt_bsp_step_workspace_bytes",
     "antdt_weighted_aggregate_backup", "antdt_aggregate_update",
     "antdt_sparse_opt_update", "antdt_dense_opt_update", "antdt_bsp_step_host", "antdt_bsp_step_device", "antdt_bsp_step_graph", "antdt_bsp_step_graph_reset",
     "antdt_read_status", "antdt_launch_count",
@@ -127,6 +128,8 @@ def lib() -> C.CDLL:
         L.antdt_embbag_bwd_dedup_static.restype = I32
         L.antdt_weighted_aggregate_workspace_bytes.argtypes = [I64, I32, I32]
         L.antdt_weighted_aggregate_workspace_bytes.restype = SZ
+        L.antdt_bsp_step_workspace_bytes.argtypes = [I64, I64, I32, I32, I64]
+        L.antdt_bsp_step_workspace_bytes.restype = SZ
         L.antdt_weighted_aggregate.argtypes = [P, P, P, I32, P, SZ, P, P]
         L.antdt_weighted_aggregate_backup.argtypes = [P, P, P, P, I32, P, SZ, P, P]
         L.antdt_weighted_aggregate_backup.restype = I32
@@ -365,6 +368,10 @@ def antdt_embbag_bwd_dedup_static(row_ids, bag_offsets, bags_per_sample: int, d_
 
 def antdt_weighted_aggregate_workspace_bytes(in_cap: int, dim: int, n_workers: int) -> int:
     return lib().antdt_weighted_aggregate_workspace_bytes(in_cap, dim, n_workers)
+
+
+def antdt_bsp_step_workspace_bytes(nnz: int, n_bags: int, dim: int, n_workers: int, uniq_cap: int) -> int:
+    return lib().antdt_bsp_step_workspace_bytes(nnz, n_bags, dim, n_workers, uniq_cap)
 
 
 def antdt_weighted_aggregate(batch_sizes: Sequence[int], ws, *, n_rows: int = 0, uniq_ids=None,

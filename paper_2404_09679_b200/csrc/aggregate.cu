@@ -363,7 +363,7 @@ void sort_merge_order(const antdt_sparse_part* sp, const uint8_t* dropped, bool 
 int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
                        const int64_t* batch_sizes, const uint8_t* dropped, int32_t n_workers,
                        void* ws, size_t ws_bytes, int32_t* dev_status, void* stream,
-                       const FusedUpdate* fu = nullptr) {
+                       const FusedUpdate* fu = nullptr, const OrderFork* fork = nullptr) {
   const int K = n_workers;
   if (K < 1 || K > kMaxSegments || !batch_sizes || !ws || !aligned16(ws)) return ANTDT_ERR_INVALID_ARG;
   double tot = 0.0;
@@ -412,12 +412,18 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
       uint32_t dropped_bits = 0;
       for (int i = 0; i < K; ++i)
         if (dropped && dropped[i]) dropped_bits |= 1u << i;
+      // the order needs the id lists only: on a forked step it runs beside the backward's sums
+      cudaStream_t so = fork ? fork->side : s;
+      if (fork && cudaStreamWaitEvent(so, fork->ids_ready, 0) != cudaSuccess) return ANTDT_ERR_CUDA;
       range_merge_order(sp->uniq_ids, sp->worker_uniq_offsets, in_cap, sp->n_rows, K, dropped_bits,
                         sp->agg_ids, sp->n_agg, agg_cap, (int64_t*)(w8 + L.wuo), bounds,
                         (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.head_bits),
                         (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap),
                         fu ? (uint32_t*)(w8 + L.row_start) : nullptr, hw, (float*)(w8 + L.weights),
-                        w8 + L.range_ws, L.range, dev_status, s);
+                        w8 + L.range_ws, L.range, dev_status, so);
+      if (fork && (cudaEventRecord(fork->order_done, so) != cudaSuccess ||
+                   cudaStreamWaitEvent(s, fork->order_done, 0) != cudaSuccess))
+        return ANTDT_ERR_CUDA;
     } else {
       sort_merge_order(sp, dropped, any_dropped, K, in_cap, agg_cap, w8, L, dev_status, s);
     }
@@ -473,6 +479,14 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
   return cuda_ok();
 }
 }  // namespace
+
+int32_t weighted_aggregate_forked(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                  const int64_t* batch_sizes, int32_t n_workers, void* ws,
+                                  size_t ws_bytes, int32_t* dev_status, void* stream,
+                                  const OrderFork* fork) {
+  return aggregate_impl(sp, dp, batch_sizes, nullptr, n_workers, ws, ws_bytes, dev_status, stream,
+                        nullptr, fork);
+}
 }  // namespace antdt
 
 extern "C" int32_t antdt_weighted_aggregate(const antdt_sparse_part* sp, const antdt_dense_part* dp,

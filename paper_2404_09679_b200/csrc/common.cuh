@@ -53,7 +53,21 @@ int32_t bwd_dedup_impl(const int32_t* row_ids, int64_t nnz, const int64_t* bag_o
                        int32_t* uniq_ids, int64_t* worker_uniq_offsets, int64_t* seg_offsets,
                        int32_t* sorted_occ, float* uniq_grads, int64_t out_cap, void* ws,
                        size_t ws_bytes, int32_t* dev_status, void* stream,
-                       const PooledArrival* arrival);  // embbag_bwd.cu
+                       const PooledArrival* arrival,
+                       cudaEvent_t ids_done = nullptr);  // embbag_bwd.cu; ids_done: recorded once the
+                                                         // distinct ids and their offsets are written
+
+// A second stream for the aggregation's merge order, which needs the workers' id lists but not
+// their gradients: the order kernels wait for ids_ready on `side`, and the caller's stream waits
+// for them (order_done) before it sums.  Used where the two chains are short enough to overlap.
+struct OrderFork {
+  cudaStream_t side;
+  cudaEvent_t ids_ready, order_done;
+};
+int32_t weighted_aggregate_forked(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                  const int64_t* batch_sizes, int32_t n_workers, void* ws,
+                                  size_t ws_bytes, int32_t* dev_status, void* stream,
+                                  const OrderFork* fork);  // aggregate.cu
 
 int32_t fwd_impl(const void* table, int32_t dtype, int64_t n_rows, int32_t dim, const int32_t* row_ids,
                  int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,

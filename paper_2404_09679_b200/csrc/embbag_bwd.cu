@@ -125,7 +125,8 @@ int32_t bwd_dedup_impl(
     int32_t bags_per_sample, const float* d_pooled, int32_t dim, int64_t n_rows, int32_t n_workers,
     const int64_t* worker_sample_offsets, int32_t* uniq_ids, int64_t* worker_uniq_offsets,
     int64_t* seg_offsets, int32_t* sorted_occ, float* uniq_grads, int64_t out_cap, void* ws,
-    size_t ws_bytes, int32_t* dev_status, void* stream, const PooledArrival* arrival) {
+    size_t ws_bytes, int32_t* dev_status, void* stream, const PooledArrival* arrival,
+    cudaEvent_t ids_done) {
   const int K = n_workers;
   if (nnz < 0 || n_bags < 0 || nnz >= (1ll << 31) || n_bags >= (1ll << 31) || n_rows < 1 ||
       n_rows >= (1ll << 31) || dim < 4 || dim > 1024 || dim % 4 || K < 1 || K > kMaxSegments ||
@@ -185,6 +186,7 @@ int32_t bwd_dedup_impl(
   segsort_runs(keys_a, nnz, uniq_ids, seg_offsets, worker_uniq_offsets, nullptr, out_cap,
                (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), tile_len, sort_ws,
                L.sort, dev_status, s);
+  if (ids_done && cudaEventRecord(ids_done, s) != cudaSuccess) return ANTDT_ERR_CUDA;
   if (nnz > 0) {
     TileArgs t;
     t.payload = occ_out;

@@ -11,15 +11,17 @@
 namespace antdt {
 // The server half of a step: aggregate, then update; in one pass when the descriptor asks for it.
 static int32_t server_step(const antdt_step_desc* d, antdt_sparse_part* sp, const antdt_dense_part* dp,
-                           void* stream) {
+                           void* stream, const OrderFork* fork = nullptr, size_t ws_skip = 0) {
   if (d->fuse_update && (d->opt == ANTDT_OPT_ADAGRAD || d->opt == ANTDT_OPT_ADAM)) {
     if (d->n_workers <= kRangeMaxWorkers) sp->agg_grads = nullptr;  // not materialised
     return antdt_aggregate_update(sp, dp, d->batch_sizes, d->n_workers, d->table, d->dtype, d->opt,
                                   d->lr, d->eps, d->beta1, d->beta2, d->step, d->state0, d->state1,
                                   d->ws, d->ws_bytes, d->d_status, stream);
   }
-  int32_t rc = antdt_weighted_aggregate(sp, dp, d->batch_sizes, d->n_workers, d->ws, d->ws_bytes,
-                                        d->d_status, stream);
+  // a forked step keeps the aggregation's scratch behind the backward's (both are live at once)
+  int32_t rc = weighted_aggregate_forked(sp, dp, d->batch_sizes, d->n_workers,
+                                         static_cast<char*>(d->ws) + ws_skip, d->ws_bytes - ws_skip,
+                                         d->d_status, stream, fork);
   if (rc != ANTDT_OK) return rc;
   return antdt_sparse_opt_update(d->table, d->dtype, d->n_rows, d->dim, d->d_agg_ids, d->d_agg_grads,
                                  d->d_n_agg, d->agg_cap, d->opt, d->lr, d->eps, d->beta1, d->beta2,
@@ -33,7 +35,9 @@ constexpr int kMaxPieces = 16;  // the d_pooled copy is cut into at most this ma
 struct StepStreams {
   bool ready = false;
   cudaStream_t in = nullptr, out = nullptr;
+  cudaStream_t side_fwd = nullptr, side_order = nullptr;  // branches of a forked device step
   cudaEvent_t start, ids, dense, fwd, done, outdone;
+  cudaEvent_t fork, fwd_done, ids_done, order_done;
   cudaEvent_t piece[kMaxPieces];
 };
 StepStreams g_ss[64];
@@ -47,7 +51,10 @@ StepStreams* step_streams() {
   if (!ss.ready) {
     if (cudaStreamCreateWithFlags(&ss.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&ss.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    cudaEvent_t* ev[] = {&ss.start, &ss.ids, &ss.dense, &ss.fwd, &ss.done, &ss.outdone};
+    if (cudaStreamCreateWithFlags(&ss.side_fwd, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&ss.side_order, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    cudaEvent_t* ev[] = {&ss.start, &ss.ids, &ss.dense, &ss.fwd, &ss.done, &ss.outdone,
+                         &ss.fork, &ss.fwd_done, &ss.ids_done, &ss.order_done};
     for (cudaEvent_t* e : ev)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     for (cudaEvent_t& e : ss.piece)
@@ -176,21 +183,57 @@ extern "C" int32_t antdt_bsp_step_host(const antdt_step_desc* d, void* stream) {
 }
 
 // The same four calls for a batch that is already resident in device memory: nothing is copied,
-// no side stream is used, the status word is left as the caller set it.
-extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream) {
+// the status word is left as the caller set it.
+//
+// forked: the step as three chains instead of one.  The forward needs nothing from the backward,
+// and the aggregation's merge order needs the workers' id lists but not their gradients, so both
+// run on side streams beside the backward (fork and join by events; in a capture they become
+// parallel branches of the graph).  It pays on small batches, where no kernel fills the device
+// and the step time is the length of the dependency chain; it needs the aggregation's scratch
+// behind the backward's instead of on top of it.
+namespace {
+constexpr int64_t kForkMaxNnz = (int64_t)1 << 22;
+
+size_t fork_ws_skip(const antdt_step_desc* d) {  // 0: no room (or no reason) to fork
+  if (d->nnz < 1 || d->nnz > kForkMaxNnz || d->fuse_update || d->n_workers > antdt::kRangeMaxWorkers ||
+      d->uniq_cap < 1)
+    return 0;
+  const size_t b = antdt_embbag_bwd_dedup_workspace_bytes(d->nnz, d->n_bags, d->dim, d->n_workers);
+  const size_t a = antdt_weighted_aggregate_workspace_bytes(d->uniq_cap, d->dim, d->n_workers);
+  const size_t skip = (b + 255) / 256 * 256;
+  if (b == 0 || a == 0 || d->ws_bytes < skip + a) return 0;
+  return skip;
+}
+
+int32_t device_step(const antdt_step_desc* d, void* stream, bool forked) {
   if (!d || d->nnz < 0 || d->n_bags < 0 || d->dim < 1 || !d->d_bag_offsets || !d->d_n_agg)
     return ANTDT_ERR_INVALID_ARG;
   const bool dense = d->d_dense_grads && d->dense_n > 0;
   if (dense && !d->d_dense_out) return ANTDT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  StepStreams* ss = nullptr;
+  size_t ws_skip = 0;
+  if (forked && (ws_skip = fork_ws_skip(d)) > 0) ss = step_streams();
+  if (!ss) ws_skip = 0;
+#define CK(x) do { if ((x) != cudaSuccess) return ANTDT_ERR_CUDA; } while (0)
+  void* fwd_stream = stream;
+  if (ss) {
+    CK(cudaEventRecord(ss->fork, s));
+    CK(cudaStreamWaitEvent(ss->side_fwd, ss->fork, 0));
+    fwd_stream = ss->side_fwd;
+  }
   int32_t rc = antdt::fwd_impl(d->table, d->dtype, d->n_rows, d->dim, d->d_row_ids, d->nnz,
-                               d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, stream,
+                               d->d_bag_offsets, d->n_bags, d->d_pooled_out, d->d_status, fwd_stream,
                                d->bags_per_sample);
-  if (rc != ANTDT_OK) return rc;
-  rc = antdt_embbag_bwd_dedup(d->d_row_ids, d->nnz, d->d_bag_offsets, d->n_bags, d->bags_per_sample,
-                              d->d_d_pooled, d->dim, d->n_rows, d->n_workers,
-                              d->worker_sample_offsets, d->d_uniq_ids, d->d_worker_uniq_offsets,
-                              d->d_seg_offsets, d->d_sorted_occ, d->d_uniq_grads, d->uniq_cap, d->ws,
-                              d->ws_bytes, d->d_status, stream);
+  if (ss) CK(cudaEventRecord(ss->fwd_done, ss->side_fwd));  // joined below even after an error
+  if (rc == ANTDT_OK)
+    rc = antdt::bwd_dedup_impl(d->d_row_ids, d->nnz, d->d_bag_offsets, d->n_bags, d->bags_per_sample,
+                               d->d_d_pooled, d->dim, d->n_rows, d->n_workers,
+                               d->worker_sample_offsets, d->d_uniq_ids, d->d_worker_uniq_offsets,
+                               d->d_seg_offsets, d->d_sorted_occ, d->d_uniq_grads, d->uniq_cap, d->ws,
+                               d->ws_bytes, d->d_status, stream, nullptr, ss ? ss->ids_done : nullptr);
+  // the update writes the table the forward reads
+  if (ss) CK(cudaStreamWaitEvent(s, ss->fwd_done, 0));
   if (rc != ANTDT_OK) return rc;
   antdt_sparse_part sp;
   sp.dim = d->dim; sp.n_rows = d->n_rows; sp.uniq_ids = d->d_uniq_ids;
@@ -199,7 +242,24 @@ extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream)
   sp.n_agg = d->d_n_agg; sp.out_cap = d->agg_cap;
   antdt_dense_part dp;
   dp.grads = d->d_dense_grads; dp.n = d->dense_n; dp.stride = d->dense_n; dp.out = d->d_dense_out;
-  return antdt::server_step(d, &sp, dense ? &dp : nullptr, stream);
+  antdt::OrderFork fork;
+  if (ss) fork = antdt::OrderFork{ss->side_order, ss->ids_done, ss->order_done};
+  return antdt::server_step(d, &sp, dense ? &dp : nullptr, stream, ss ? &fork : nullptr, ws_skip);
+#undef CK
+}
+}  // namespace
+
+extern "C" int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream) {
+  return device_step(d, stream, false);
+}
+
+extern "C" size_t antdt_bsp_step_workspace_bytes(int64_t nnz, int64_t n_bags, int32_t dim,
+                                                 int32_t n_workers, int64_t uniq_cap) {
+  const size_t b = antdt_embbag_bwd_dedup_workspace_bytes(nnz, n_bags, dim, n_workers);
+  const size_t a = antdt_weighted_aggregate_workspace_bytes(uniq_cap, dim, n_workers);
+  if (b == 0 || a == 0) return 0;
+  if (nnz <= kForkMaxNnz && n_workers <= antdt::kRangeMaxWorkers) return (b + 255) / 256 * 256 + a;
+  return b > a ? b : a;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -292,7 +352,7 @@ extern "C" int32_t antdt_bsp_step_graph(const antdt_step_desc* d, void* stream) 
   }
   const int64_t before = antdt_launch_count();
   antdt::prof_untimed(true);
-  const int32_t rc = antdt_bsp_step_device(d, stream);
+  const int32_t rc = device_step(d, stream, true);  // forked where the descriptor allows it
   antdt::prof_untimed(false);
   const int64_t n_kernels = antdt_launch_count() - before;
   antdt::count_launches(-n_kernels);  // captured, not run

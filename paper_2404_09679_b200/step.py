@@ -44,8 +44,7 @@ class StepBuffers:
         self.n_agg = torch.zeros(1, dtype=i64, device=dev)
         self.status = torch.zeros(1, dtype=i32, device=dev)
         self.dense_out = torch.empty(dense_n, dtype=f32, device=dev) if dense_n else None
-        ws_bytes = max(B.antdt_embbag_bwd_dedup_workspace_bytes(max_nnz, max_bags, dim, n_workers),
-                       B.antdt_weighted_aggregate_workspace_bytes(self.uniq_cap, dim, n_workers))
+        ws_bytes = B.antdt_bsp_step_workspace_bytes(max_nnz, max_bags, dim, n_workers, self.uniq_cap)
         self.ws = torch.empty((ws_bytes + 255) // 256 * 256, dtype=torch.uint8, device=dev)
 
 

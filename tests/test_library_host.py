@@ -67,6 +67,16 @@ def test_device_calls_reject_bad_arguments_before_any_launch():
     assert B.antdt_launch_count() == n0
     assert B.antdt_weighted_aggregate_workspace_bytes(100, 16, 4) > 0
     assert B.antdt_weighted_aggregate_workspace_bytes(100, 16, 2000) == 0
+    # a step's workspace: room for both scratch areas side by side on a small batch (the
+    # three-branch graph), the larger of the two on a large one, 0 when either figure is 0
+    b = B.antdt_embbag_bwd_dedup_workspace_bytes(1000, 100, 16, 4)
+    a = B.antdt_weighted_aggregate_workspace_bytes(1000, 16, 4)
+    assert B.antdt_bsp_step_workspace_bytes(1000, 100, 16, 4, 1000) == (b + 255) // 256 * 256 + a
+    big = 1 << 23
+    b = B.antdt_embbag_bwd_dedup_workspace_bytes(big, big, 16, 4)
+    a = B.antdt_weighted_aggregate_workspace_bytes(big, 16, 4)
+    assert B.antdt_bsp_step_workspace_bytes(big, big, 16, 4, big) == max(a, b)
+    assert B.antdt_bsp_step_workspace_bytes(1000, 100, 16, 2000, 1000) == 0
 
 
 # ---- planner: library vs checker, bit for bit ---------------------------------------------
