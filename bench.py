@@ -623,6 +623,10 @@ def run_ours(args):
             "value": e2e_samples / (e2e_ms * 1e-3), "unit": UNIT,
             "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
             "ms_per_step": e2e_ms / K_steps,
+            "h2d_GBps": round(e2e["h2d"] / (e2e_ms / K_steps * 1e-3) / 1e9, 2),
+            "link": e2e.get("link"),
+            "frac_of_link": (round(e2e["h2d"] / (e2e_ms / K_steps * 1e-3) / 1e9 /
+                                   e2e["link"]["h2d_beside_d2h_GBps"], 4) if e2e.get("link") else None),
             "how": "antdt_bsp_step_host, two staging sets alternated: the copies of step s+1 run "
                    "under the kernels of step s; the host reads every step's results"},
         "gpu_launches": launches,
@@ -723,7 +727,38 @@ def run_e2e(B, w, batches, buf, table, state0, state1, oc, W, K_steps, dev, stre
     h2d = (b["ids"].numel() * 4 + b["off"].numel() * 8 + b["dY"].numel() * 4 +
            (b["dense"].numel() * 4 if b["dense"] is not None else 0))
     d2h = (b["off"].numel() - 1) * w.D * 4 + w.dense_n * 4 + 12
-    return {"ms": e0.elapsed_time(e1), "samples": samples, "h2d": h2d, "d2h": d2h}
+    return {"ms": e0.elapsed_time(e1), "samples": samples, "h2d": h2d, "d2h": d2h,
+            "link": measure_link(host[0]["dY"], sets[0], stream)}
+
+
+def measure_link(h_src, st, stream):
+    """The host link the end-to-end step rides on: the largest input copied host-to-device alone,
+    then with the largest result going device-to-host at the same time (as in a step).  Plain
+    cudaMemcpyAsync through torch, page-locked on the host side; GB/s of the host-to-device copy."""
+    n = min(h_src.numel(), st.d_d_pooled.numel(), st.h_pooled.numel())
+    if n * 4 < (1 << 20):
+        return None
+    src, dst = h_src.reshape(-1)[:n], st.d_d_pooled.reshape(-1)[:n]
+    back_src, back_dst = st.d_pooled_out.reshape(-1)[:n], st.h_pooled.reshape(-1)[:n]
+    side = torch.cuda.Stream()
+    out = {}
+    for name, both in (("h2d_alone_GBps", False), ("h2d_beside_d2h_GBps", True)):
+        best = 0.0
+        for _ in range(3):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if both:
+                with torch.cuda.stream(side):
+                    back_dst.copy_(back_src, non_blocking=True)
+                    back_dst.copy_(back_src, non_blocking=True)   # still running when the other ends
+            with torch.cuda.stream(stream):
+                e0.record(stream)
+                dst.copy_(src, non_blocking=True)
+                e1.record(stream)
+            torch.cuda.synchronize()
+            best = max(best, n * 4 / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+        out[name] = round(best, 2)
+    return out
 
 
 # ------------------------------------------------------------------------------------------
