@@ -244,6 +244,21 @@ range_scan_kernel(const int32_t* __restrict__ distinct, int64_t P, int64_t* __re
 // Shared memory: mask[R] (worker set per row id), pres[R/32] (presence bits: the table is
 // sparse, so everything after the fill walks presence words and present ids only), per presence
 // word the present ids before it (wrank), per present id the contributions before it (first_c).
+// The worker sets are as wide as the worker count needs (8, 16 or 32 bits, packed into words) and
+// first_c is 16 bits wide when a range cannot hold more than 2^16 entries: a CTA's shared memory
+// decides how many ranges an SM works on at once, and with few entries per range the kernel's
+// time is the number of CTA waves times a CTA's chain of global round trips.
+struct EmitShape {
+  int mask_lg;  // worker sets per 32-bit word, log2: 0, 1 (up to 16 workers), 2 (up to 8)
+  int fc16;     // first_c holds 16-bit values
+};
+__host__ __device__ inline EmitShape emit_shape(int r_log2, int K) {
+  EmitShape e;
+  e.mask_lg = K <= 8 ? 2 : (K <= 16 ? 1 : 0);
+  e.fc16 = ((int64_t)K << r_log2) <= 65536 ? 1 : 0;
+  return e;
+}
+
 __global__ void __launch_bounds__(kRaThreads)
 range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ bnd,
                   const int64_t* __restrict__ wuo, int K, int64_t P, int r_log2, int64_t n_rows,
@@ -254,9 +269,14 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   extern __shared__ __align__(16) unsigned char ra_smem[];
   const int R = 1 << r_log2;
   const int nW = R / 32;  // presence words: at most 256 = one per thread
-  uint32_t* mask = reinterpret_cast<uint32_t*>(ra_smem);
-  uint32_t* first_c = mask + R;
-  int64_t* s_before = reinterpret_cast<int64_t*>(first_c + R);
+  const EmitShape shp = emit_shape(r_log2, K);
+  const int lg = shp.mask_lg, sub = (1 << lg) - 1, sub_sh = 5 - lg;
+  const uint32_t set_bits = 0xffffffffu >> (32 - (32 >> lg));
+  uint32_t* mask = reinterpret_cast<uint32_t*>(ra_smem);  // R >> lg words
+  uint32_t* first_c = mask + (R >> lg);
+  unsigned short* first_c16 = reinterpret_cast<unsigned short*>(first_c);
+  int64_t* s_before = reinterpret_cast<int64_t*>(first_c + (shp.fc16 ? R / 2 : R));
+  auto workers_of = [&](int kl) { return (mask[kl >> lg] >> ((kl & sub) << sub_sh)) & set_bits; };
   uint32_t* pres = reinterpret_cast<uint32_t*>(s_before + 1);  // [256]
   int32_t* wrank = reinterpret_cast<int32_t*>(pres + 256);     // [256]
   int32_t* s_beg = wrank + 256;  // [32]
@@ -282,13 +302,13 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   if (tid < nW) pres[tid] = 0u;
   {
     uint4* m4 = reinterpret_cast<uint4*>(mask);
-    for (int i = tid; i < R / 4; i += kRaThreads) m4[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < (R >> lg) / 4; i += kRaThreads) m4[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   __syncthreads();
   const uint32_t base_key = (uint32_t)(b << r_log2);
   for_each_entry(ids, pc.entries, R, base_key, n_rows, s_beg, s_off, status,
                  [&](int w, int, uint32_t, uint32_t kl) {
-                   atomicOr(&mask[kl], 1u << w);
+                   atomicOr(&mask[kl >> lg], (1u << w) << ((kl & sub) << sub_sh));
                    atomicOr(&pres[kl >> 5], 1u << (kl & 31));
                  });
   __syncthreads();
@@ -296,16 +316,17 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   // thread q owns presence word q: present ids and contributions in it, prefix sums over the words
   const uint32_t pw = tid < nW ? pres[tid] : 0u;
   int n_ids = __popc(pw), n_con = 0;
-  for (uint32_t rest = pw; rest; rest &= rest - 1u) n_con += __popc(mask[tid * 32 + __ffs((int)rest) - 1]);
+  for (uint32_t rest = pw; rest; rest &= rest - 1u) n_con += __popc(workers_of(tid * 32 + __ffs((int)rest) - 1));
   int tot_ids, tot_con;
   block_scan2(n_ids, n_con, tot_ids, tot_con, s_tmp);  // now exclusive prefixes
   if (tid < nW) {
     wrank[tid] = n_ids;
     int t = n_ids, first = n_con;
     for (uint32_t rest = pw; rest; rest &= rest - 1u) {
-      first_c[t++] = (uint32_t)first;
+      if (shp.fc16) first_c16[t++] = (unsigned short)first;
+      else first_c[t++] = (uint32_t)first;
       atomicOr(&hb[(hb_shift + first) >> 5], 1u << ((hb_shift + first) & 31));
-      first += __popc(mask[tid * 32 + __ffs((int)rest) - 1]);
+      first += __popc(workers_of(tid * 32 + __ffs((int)rest) - 1));
     }
   }
   __syncthreads();
@@ -322,8 +343,8 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   for_each_entry(ids, pc.entries, R, base_key, n_rows, s_beg, s_off, nullptr,
                  [&](int w, int j, uint32_t id, uint32_t kl) {
                    const int t = wrank[kl >> 5] + __popc(pres[kl >> 5] & ((1u << (kl & 31)) - 1u));
-                   const int slot = __popc(mask[kl] & ((1u << w) - 1u));
-                   const int64_t dest = pc.before + (int64_t)first_c[t] + slot;
+                   const int slot = __popc(workers_of((int)kl) & ((1u << w) - 1u));
+                   const int64_t dest = pc.before + (int64_t)(shp.fc16 ? first_c16[t] : first_c[t]) + slot;
                    const int64_t u = u0 + t;
                    src[dest] = (uint32_t)j;
                    if (slot == 0 && u < out_cap) {
@@ -336,7 +357,9 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
 
 size_t emit_smem(int r_log2, int K) {  // tables, small arrays, head bits of up to R*K slots
   const size_t R = (size_t)1 << r_log2;
-  return 8 * R + 8 + 4 * (256 + 256 + 32 + 33 + 16) + 4 * (R * (size_t)K / 32 + 2) + 12;
+  const EmitShape e = emit_shape(r_log2, K);
+  return 4 * (R >> e.mask_lg) + (e.fc16 ? 2 : 4) * R + 8 + 4 * (256 + 256 + 32 + 33 + 16) +
+         4 * (R * (size_t)K / 32 + 2) + 12;
 }
 
 }  // namespace
