@@ -354,7 +354,7 @@ void sort_merge_order(const antdt_sparse_part* sp, const uint8_t* dropped, bool 
     }
     segsort_setup(bounds, 1, in_cap, sort_ws, L.sort, s);
     segsort_run(sort_keys, sort_vals, keys_a, (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.keys_b),
-                (uint32_t*)(w8 + L.vals_t), key_bits, 0, sort_ws, L.sort, dev_status, s, true);
+                (uint32_t*)(w8 + L.vals_t), key_bits, 0, in_cap, sort_ws, L.sort, dev_status, s, true);
     segsort_runs(keys_a, in_cap, sp->agg_ids, (int64_t*)(w8 + L.run_start), nullptr, sp->n_agg,
                  agg_cap, (uint32_t*)(w8 + L.head_bits),
                  (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap > 0 ? in_cap : 1), sort_ws, L.sort, dev_status, s, true);

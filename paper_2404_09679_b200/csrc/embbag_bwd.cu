@@ -182,7 +182,7 @@ int32_t bwd_dedup_impl(
                  expand_to, dev_status);
   }
   segsort_run(reinterpret_cast<const uint32_t*>(row_ids), expand_to, keys_a, occ_out, keys_b,
-              vals_t, key_bits, n_rows, sort_ws, L.sort, dev_status, s);
+              vals_t, key_bits, n_rows, nnz, sort_ws, L.sort, dev_status, s);
   segsort_runs(keys_a, nnz, uniq_ids, seg_offsets, worker_uniq_offsets, nullptr, out_cap,
                (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), tile_len, sort_ws,
                L.sort, dev_status, s);

@@ -261,6 +261,7 @@ radix_scan_kernel(const SortDesc* __restrict__ desc, const int32_t* __restrict__
 // counters over the warps and over the bins -> reorder the tile in shared memory -> write
 // every bin's run to its global slot with consecutive threads.
 // ---------------------------------------------------------------------------------------
+constexpr int kFoldScanChunks = 128;  // up to this many chunks the scatter scans the counts itself
 constexpr int kScatThreads = 512;
 constexpr int kScatItems = kSortTile / kScatThreads;  // 8
 constexpr int kScatWarps = kScatThreads / 32;         // 16
@@ -272,7 +273,8 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
                      uint32_t mask, const SortDesc* __restrict__ desc,
                      const int32_t* __restrict__ chunk_seg, const int64_t* __restrict__ seg_bounds,
                      const int64_t* __restrict__ chunk_begin, const int64_t* __restrict__ chunk_end,
-                     const uint32_t* __restrict__ hist, const uint32_t* __restrict__ bin_base) {
+                     const uint32_t* __restrict__ hist, const uint32_t* __restrict__ bin_base,
+                     const int32_t* __restrict__ seg_first) {
   const int c = blockIdx.x;
   if (c >= desc->n_chunks) return;
   extern __shared__ __align__(16) unsigned char scat_smem[];
@@ -287,7 +289,38 @@ radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __res
   const unsigned lt = (1u << lane) - 1u;
   const int seg = chunk_seg[c];
   const uint32_t seg_begin = (uint32_t)seg_bounds[seg];
-  gbase[tid] = seg_begin + bin_base[(size_t)seg * kSortMaxBins + tid] + hist[(size_t)c * kSortMaxBins + tid];
+  if (seg_first) {
+    // few chunks (a small input): `hist` holds the raw counts and this CTA sums its segment's
+    // chunks itself - bin totals, the part before its own chunk, the scan over the bins - which
+    // costs a microsecond and saves the scan kernel between the histogram and this one
+    const int c0 = seg_first[seg], c1 = seg_first[seg + 1];
+    uint32_t pre = 0, tot = 0;
+    for (int cc = c0; cc < c1; cc += 4) {
+      uint32_t h[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) h[j] = cc + j < c1 ? hist[(size_t)(cc + j) * kSortMaxBins + tid] : 0u;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        pre += cc + j < c ? h[j] : 0u;
+        tot += h[j];
+      }
+    }
+    uint32_t incl = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[w] = incl;
+    __syncthreads();
+    uint32_t wp = 0;
+#pragma unroll
+    for (int ww = 0; ww < kScatWarps; ++ww) wp += (ww < w) ? warp_tot[ww] : 0u;
+    gbase[tid] = seg_begin + (incl - tot + wp) + pre;
+    // warp_tot is written again only after the tile loop's barriers (A) and (B)
+  } else {
+    gbase[tid] = seg_begin + bin_base[(size_t)seg * kSortMaxBins + tid] + hist[(size_t)c * kSortMaxBins + tid];
+  }
   unsigned short* my_wh = wh + w * kSortMaxBins;
 
   const int64_t cb = chunk_begin[c], ce = chunk_end[c];
@@ -634,9 +667,16 @@ void segsort_prepare_device() {
   done = true;
 }
 
+// Chunks the set-up can have cut for n_cap elements: a chunk holds at least one tile, and every
+// segment may end in a partial one.
+static int chunk_bound(int64_t n_cap, const SortLayout& L) {
+  const int64_t c = (n_cap > 0 ? n_cap : 0) / kSortTile + L.n_segments + 1;
+  return (int)(c < L.max_chunks ? c : L.max_chunks);
+}
+
 void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* keys_out,
                  uint32_t* vals_out, uint32_t* keys_tmp, uint32_t* vals_tmp, int key_bits,
-                 int64_t check_rows, char* ws, const SortLayout& L, int32_t* status,
+                 int64_t check_rows, int64_t n_cap, char* ws, const SortLayout& L, int32_t* status,
                  cudaStream_t s, bool agg) {
   const SortDesc* desc = (const SortDesc*)(ws + L.desc);
   const int64_t* seg_bounds = (const int64_t*)(ws + L.seg_bounds);
@@ -662,11 +702,14 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
     uint32_t* vout = to_out ? vals_out : vals_tmp;
     ANTDT_LAUNCH(agg ? "agg_radix_hist" : "radix_hist", radix_hist_kernel, L.max_chunks, kHistThreads, 0, s, kin, shift,
                  mask, desc, chunk_begin, chunk_end, hist, p == 0 ? check_rows : (int64_t)0, status);
-    ANTDT_LAUNCH(agg ? "agg_radix_scan" : "radix_scan", radix_scan_kernel, S, kSortMaxBins, 0, s, desc, seg_first, hist,
-                 bin_base);
+    // with few chunks every scatter CTA scans the counts it needs itself (one launch less)
+    const bool fold_scan = chunk_bound(n_cap, L) <= kFoldScanChunks;
+    if (!fold_scan)
+      ANTDT_LAUNCH(agg ? "agg_radix_scan" : "radix_scan", radix_scan_kernel, S, kSortMaxBins, 0, s, desc, seg_first, hist,
+                   bin_base);
     ANTDT_LAUNCH(agg ? "agg_radix_scatter" : "radix_scatter", radix_scatter_kernel, L.max_chunks, kScatThreads, kScatSmem, s, kin, vin,
                  kout, vout, shift, mask, desc, chunk_seg, seg_bounds, chunk_begin, chunk_end, hist,
-                 bin_base);
+                 bin_base, fold_scan ? seg_first : (const int32_t*)nullptr);
     kin = kout;
     vin = vout;
     shift += bits;

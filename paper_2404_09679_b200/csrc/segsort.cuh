@@ -80,10 +80,11 @@ bool segsort_setup_workers(const int64_t* wso_host, int n_workers, int bags_per_
 // Sorts by the low key_bits bits.  keys_in is read only; the sorted pairs land in
 // keys_out/vals_out; keys_tmp/vals_tmp are scratch of the same size.  vals_in == nullptr means
 // "value = element index".  check_rows > 0: keys >= check_rows raise ID_OUT_OF_RANGE.
+// n_cap: the element count the set-up was given (a host-side bound on the chunks that exist).
 // agg only selects the names under which the launches are accounted.
 void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* keys_out,
                  uint32_t* vals_out, uint32_t* keys_tmp, uint32_t* vals_tmp, int key_bits,
-                 int64_t check_rows, char* ws, const SortLayout& L, int32_t* status,
+                 int64_t check_rows, int64_t n_cap, char* ws, const SortLayout& L, int32_t* status,
                  cudaStream_t s, bool agg = false);
 
 // Runs of equal keys inside the segments of a sorted array.
