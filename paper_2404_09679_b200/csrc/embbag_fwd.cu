@@ -1,10 +1,15 @@
 // Worker forward: embedding-bag gather with sum pooling.
 //
 // One group of G lanes owns one bag; a row is read as G (x VPL) 16-byte vectors, so a warp
-// issues fully coalesced 128-bit loads over 32/G rows at once.  The bag's id list is staged
-// through the group's registers G ids at a time (one coalesced load, then shuffles), and U row
-// loads are put in flight before any is consumed.  The path is a random gather bound by HBM
-// (hot rows by L2); there is no contraction here and so no tensor-core work.
+// issues fully coalesced 128-bit loads over 32/G rows at once.  The path is a random gather bound
+// by the latency of its chain of dependent loads (offsets -> ids -> rows) and by HBM / L2 for the
+// rows; there is no contraction here and so no tensor-core work.  Three kernels:
+//   embbag_fwd_flat_kernel    rows of up to 512 bytes, one bag per group: every lane reads the ids
+//                             itself, four rows in flight, 32 registers -> 64 warps per SM
+//   embbag_fwd_stride_kernel  the same for short bags: capped grid, groups stride over the bags
+//                             and read the next bag's offsets ahead
+//   embbag_fwd_kernel         wider rows (VPL vectors per lane): ids staged through the group's
+//                             registers G at a time (one coalesced load, then shuffles)
 #include "common.cuh"
 
 namespace antdt {
@@ -108,11 +113,194 @@ embbag_fwd_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
   }
 }
 
+
+// The gather with the plainest possible inner loop, for rows of up to 512 bytes: every lane
+// reads the bag's ids itself (the G lanes of a group ask for the same address: one transaction),
+// four row loads are requested before any is consumed, nothing is exchanged between lanes, and
+// the register budget (32) lets 64 warps share an SM.  What bounds this kernel is the chain
+// offsets -> ids -> rows of dependent loads, and only the number of warps in flight hides it:
+// eight loads per lane at 48 or 40 warps per SM were slower on every workload measured.
+constexpr int kFlatThreads = 256;
+constexpr int kFlatUnroll = 4;
+constexpr int kFlatCtas = 8;     // CTAs per SM
+constexpr int kFlatWaves = 32;   // grid cap of the striding form, in resident waves
+
+// One bag: this lane's 16 bytes of the sum of the rows that ids[0..len) name, as packed fp32 pairs.
+// (The output address is formed by the caller after the loop: at 32 registers every 64-bit value
+// that lives across the loop costs loads in flight.)
+template <int G, bool BF16>
+__device__ __forceinline__ void flat_bag(const uint4* __restrict__ tbl, uint32_t row_vecs, uint32_t limit,
+                                         const int32_t* __restrict__ ids, int len, int lg, bool lane_on,
+                                         uint64_t (&acc)[BF16 ? 4 : 2], bool& bad) {
+  constexpr int PAIRS = BF16 ? 4 : 2;
+#pragma unroll
+  for (int e = 0; e < PAIRS; ++e) acc[e] = 0ull;
+  for (int j0 = 0; j0 < len; j0 += kFlatUnroll) {
+    uint4 v[kFlatUnroll];
+#pragma unroll
+    for (int t = 0; t < kFlatUnroll; ++t) {
+      const bool in = j0 + t < len;
+      const uint32_t id = in ? (uint32_t)__ldg(ids + j0 + t) : 0u;
+      const bool ok = in && id < limit;
+      bad |= in && !ok;  // skipped: contributes nothing
+      v[t] = (ok && lane_on) ? __ldg(tbl + (size_t)id * row_vecs + lg) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int t = 0; t < kFlatUnroll; ++t) {
+      if (BF16) {  // bf16 -> fp32 is a 16-bit shift; a zero vector adds +0.0
+        acc[0] = f32x2_add(acc[0], f32x2_pack(v[t].x << 16, v[t].x & 0xffff0000u));
+        acc[1] = f32x2_add(acc[1], f32x2_pack(v[t].y << 16, v[t].y & 0xffff0000u));
+        acc[2] = f32x2_add(acc[2], f32x2_pack(v[t].z << 16, v[t].z & 0xffff0000u));
+        acc[3] = f32x2_add(acc[3], f32x2_pack(v[t].w << 16, v[t].w & 0xffff0000u));
+      } else {
+        acc[0] = f32x2_add(acc[0], f32x2_pack(v[t].x, v[t].y));
+        acc[1] = f32x2_add(acc[1], f32x2_pack(v[t].z, v[t].w));
+      }
+    }
+  }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void flat_store(float* __restrict__ out, const uint64_t (&acc)[BF16 ? 4 : 2]) {
+  ulonglong2* o = reinterpret_cast<ulonglong2*>(out);
+  o[0] = make_ulonglong2(acc[0], acc[1]);
+  if (BF16) o[1] = make_ulonglong2(acc[2], acc[3]);
+}
+
+// A bag's id range; bad offsets are flagged and read as an empty bag.
+__device__ __forceinline__ void flat_range(const int64_t* __restrict__ bag_offsets, int64_t bag, int64_t nnz,
+                                           int lg, int32_t* status, int32_t& begin, int32_t& len) {
+  const int64_t b = bag_offsets[bag], e = bag_offsets[bag + 1];
+  begin = 0;
+  len = 0;
+  if (b < 0 || e < b || e > nnz) {
+    if (lg == 0) set_status(status, ANTDT_ERR_BAD_OFFSETS);
+    return;
+  }
+  begin = (int32_t)b;  // nnz < 2^31
+  len = (int32_t)(e - b);
+}
+
+// One bag per lane group.  BY_FIELD: a CTA takes the bags of ONE field of consecutive samples and
+// consecutive CTAs stay on that field (bag = sample * fields + field), so that what is resident
+// on an SM and in L2 at one time draws from one field's hot rows.
+template <int G, bool BF16, bool BY_FIELD>
+__global__ void __launch_bounds__(kFlatThreads, kFlatCtas)
+embbag_fwd_flat_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
+                       const int32_t* __restrict__ row_ids, int64_t nnz,
+                       const int64_t* __restrict__ bag_offsets, int64_t n_bags,
+                       float* __restrict__ pooled, int32_t* status, int fields, int64_t sample_blocks) {
+  constexpr int EPV = BF16 ? 8 : 4;
+  const int lg = threadIdx.x & (G - 1);
+  int64_t bag;
+  if (BY_FIELD) {
+    const int64_t f = blockIdx.x / sample_blocks, sb = blockIdx.x % sample_blocks;
+    bag = (sb * (kFlatThreads / G) + (threadIdx.x / G)) * fields + f;
+  } else {
+    bag = (int64_t)blockIdx.x * (kFlatThreads / G) + (threadIdx.x / G);
+  }
+  if (bag >= n_bags) return;
+  const int nvec = dim / EPV;
+  int32_t begin, len;
+  flat_range(bag_offsets, bag, nnz, lg, status, begin, len);
+  bool bad = false;
+  uint64_t acc[BF16 ? 4 : 2];
+  flat_bag<G, BF16>(static_cast<const uint4*>(table), (uint32_t)nvec, (uint32_t)n_rows, row_ids + begin, len,
+                    lg, lg < nvec, acc, bad);
+  if (bad) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
+  if (lg < nvec) flat_store<BF16>(pooled + bag * (int64_t)dim + (size_t)lg * EPV, acc);
+}
+
+// Short bags (a few ids each): the chain offsets -> ids -> rows is most of a bag's time, so the
+// grid is capped, every lane group strides over its bags (bag order), and the NEXT bag's offsets
+// are read before the current bag's rows are requested (30 fields x 4.5 ids x 128-byte rows:
+// 1.06 -> 0.84 ms).  The loop is written out in one piece on purpose: at 32 registers the form of
+// the source decides what the compiler keeps in flight, and two tidier versions of this same loop
+// (the bag's sum in a helper, the offsets held as raw 64-bit values) measured 1.07 - 1.21 ms.
+template <int G, bool BF16>
+__global__ void __launch_bounds__(kFlatThreads, kFlatCtas)
+embbag_fwd_stride_kernel(const void* __restrict__ table, int64_t n_rows, int dim,
+                         const int32_t* __restrict__ row_ids, int64_t nnz,
+                         const int64_t* __restrict__ bag_offsets, int64_t n_bags,
+                         float* __restrict__ pooled, int32_t* status) {
+  constexpr int EPV = BF16 ? 8 : 4;
+  constexpr int PAIRS = EPV / 2;
+  constexpr int GPB = kFlatThreads / G;  // groups (bags) per CTA and turn
+  const int lg = threadIdx.x & (G - 1);
+  const int nvec = dim / EPV;
+  const uint32_t limit = (uint32_t)n_rows;
+  const bool lane_on = lg < nvec;
+  const uint4* tbl = static_cast<const uint4*>(table);
+  const uint32_t row_vecs = (uint32_t)nvec;
+  // 32-bit bag numbers: there are fewer than 2^31 bags
+  const uint32_t n_slots = (uint32_t)n_bags;
+  const uint32_t stride = gridDim.x * GPB;
+  auto range_of = [&](uint32_t q, int32_t& bg, int32_t& b0, int32_t& ln) {
+    bg = -1; b0 = 0; ln = 0;
+    if (q >= n_slots) return;
+    bg = (int32_t)q;
+    const int64_t begin = bag_offsets[q], end = bag_offsets[q + 1];
+    if (begin < 0 || end < begin || end > nnz) {
+      if (lg == 0) set_status(status, ANTDT_ERR_BAD_OFFSETS);
+      return;
+    }
+    b0 = (int32_t)begin;  // nnz < 2^31
+    ln = (int32_t)(end - begin);
+  };
+  uint32_t q = blockIdx.x * GPB + threadIdx.x / G;
+  int32_t bag, begin, len;
+  range_of(q, bag, begin, len);
+  bool bad = false;
+  while (q < n_slots) {
+    // the next turn's offsets are requested before this turn's rows
+    int32_t nbag, nbegin, nlen;
+    range_of(q + stride < q ? n_slots : q + stride, nbag, nbegin, nlen);
+    if (bag >= 0) {
+      const int32_t* ids = row_ids + begin;
+      uint64_t acc[PAIRS];
+#pragma unroll
+      for (int e = 0; e < PAIRS; ++e) acc[e] = 0ull;
+      for (int j0 = 0; j0 < len; j0 += kFlatUnroll) {
+        uint4 v[kFlatUnroll];
+#pragma unroll
+        for (int t = 0; t < kFlatUnroll; ++t) {
+          const bool in = j0 + t < len;
+          const uint32_t id = in ? (uint32_t)__ldg(ids + j0 + t) : 0u;
+          const bool ok = in && id < limit;
+          bad |= in && !ok;
+          v[t] = (ok && lane_on) ? __ldg(tbl + (size_t)id * row_vecs + lg) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int t = 0; t < kFlatUnroll; ++t) {
+          if (BF16) {
+            acc[0] = f32x2_add(acc[0], f32x2_pack(v[t].x << 16, v[t].x & 0xffff0000u));
+            acc[1] = f32x2_add(acc[1], f32x2_pack(v[t].y << 16, v[t].y & 0xffff0000u));
+            acc[2] = f32x2_add(acc[2], f32x2_pack(v[t].z << 16, v[t].z & 0xffff0000u));
+            acc[3] = f32x2_add(acc[3], f32x2_pack(v[t].w << 16, v[t].w & 0xffff0000u));
+          } else {
+            acc[0] = f32x2_add(acc[0], f32x2_pack(v[t].x, v[t].y));
+            acc[1] = f32x2_add(acc[1], f32x2_pack(v[t].z, v[t].w));
+          }
+        }
+      }
+      if (lane_on) {
+        ulonglong2* o = reinterpret_cast<ulonglong2*>(pooled + bag * (int64_t)dim + (size_t)lg * EPV);
+        o[0] = make_ulonglong2(acc[0], acc[1]);
+        if (BF16) o[1] = make_ulonglong2(acc[2], acc[3]);
+      }
+    }
+    if (q + stride < q) break;  // wrapped: nothing further
+    q += stride; bag = nbag; begin = nbegin; len = nlen;
+  }
+  if (bad) set_status(status, ANTDT_ERR_ID_OUT_OF_RANGE);
+}
+
 template <int G, int VPL, bool BF16>
 void launch_fwd(const void* table, int64_t n_rows, int dim, const int32_t* row_ids, int64_t nnz,
                 const int64_t* bag_offsets, int64_t n_bags, float* pooled, int32_t* status,
-                cudaStream_t s, int fields) {
-  const int64_t gpb = kFwdThreads / G;
+                cudaStream_t s, int fields, bool short_bags) {
+  constexpr bool flat = VPL == 1;  // rows of up to 512 bytes
+  const int64_t gpb = (flat ? kFlatThreads : kFwdThreads) / G;
   int64_t grid = (n_bags + gpb - 1) / gpb, sample_blocks = 0;
   if (fields > 0 && n_bags % fields == 0) {
     sample_blocks = (n_bags / fields + gpb - 1) / gpb;
@@ -120,21 +308,33 @@ void launch_fwd(const void* table, int64_t n_rows, int dim, const int32_t* row_i
   } else {
     fields = 0;
   }
-  if (fields > 0)
+  if (flat && short_bags) {
+    const int64_t cap = (int64_t)kNumSM * kFlatCtas * kFlatWaves;
+    grid = (n_bags + gpb - 1) / gpb;
+    ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_stride_kernel<G, BF16>), (unsigned)(grid < cap ? grid : cap),
+                 kFlatThreads, 0, s, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status);
+  } else if (flat && fields > 0) {
+    ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_flat_kernel<G, BF16, true>), (unsigned)grid, kFlatThreads, 0, s,
+                 table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status, fields, sample_blocks);
+  } else if (flat) {
+    ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_flat_kernel<G, BF16, false>), (unsigned)grid, kFlatThreads, 0, s,
+                 table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status, fields, sample_blocks);
+  } else if (fields > 0) {
     ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_kernel<G, VPL, BF16, true>), (unsigned)grid, kFwdThreads, 0, s,
                  table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status, fields, sample_blocks);
-  else
+  } else {
     ANTDT_LAUNCH("embbag_fwd", (embbag_fwd_kernel<G, VPL, BF16, false>), (unsigned)grid, kFwdThreads, 0, s,
                  table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled, status, fields, sample_blocks);
+  }
 }
 
 template <bool BF16>
 int32_t dispatch_fwd(int nvec, const void* table, int64_t n_rows, int dim, const int32_t* row_ids,
                      int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,
-                     int32_t* status, cudaStream_t s, int fields) {
+                     int32_t* status, cudaStream_t s, int fields, bool short_bags) {
 #define FWD_CASE(G, VPL)                                                                      \
   launch_fwd<G, VPL, BF16>(table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,     \
-                           status, s, fields);                                                \
+                           status, s, fields, short_bags);                                    \
   return ANTDT_OK;
   if (nvec <= 1) { FWD_CASE(1, 1) }
   if (nvec <= 2) { FWD_CASE(2, 1) }
@@ -169,14 +369,15 @@ int32_t fwd_impl(const void* table, int32_t dtype, int64_t n_rows, int32_t dim, 
   // Field-major order pays when a bag's id list fills a 32-byte sector (eight ids or more on
   // average): measured -12% on 100 fields x 10 ids x 256-byte rows, -2% on 40 x 20 x 128-byte rows,
   // but +8% on 30 fields x 4.5 ids, where the scattered id reads cost more than the rows gain.
-  const int fields = (bags_per_sample > 1 && nnz >= 8 * n_bags) ? bags_per_sample : 0;
+  const bool short_bags = nnz < 8 * n_bags;
+  const int fields = (bags_per_sample > 1 && !short_bags) ? bags_per_sample : 0;
   int32_t rc;
   if (dtype == ANTDT_BF16)
     rc = dispatch_fwd<true>(dim / 8, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags, pooled,
-                            dev_status, s, fields);
+                            dev_status, s, fields, short_bags);
   else
     rc = dispatch_fwd<false>(dim / 4, table, n_rows, dim, row_ids, nnz, bag_offsets, n_bags,
-                             pooled, dev_status, s, fields);
+                             pooled, dev_status, s, fields, short_bags);
   if (rc != ANTDT_OK) return rc;
   return cuda_ok();
 }
