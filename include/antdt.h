@@ -440,7 +440,7 @@ int32_t antdt_bsp_step_device(const antdt_step_desc* d, void* stream);
  *     executables are driver objects, the only thing this library ever creates on a device.
  *   - Per-kernel event timing (antdt_profile_enable) does not see kernels inside a graph;
  *     antdt_launch_count counts a replay's kernel nodes.
- *   - Small batches (at most 2^22 occurrences, at most 32 workers, no fuse_update) are captured
+ *   - Small batches (at most 2^22 occurrences, at most 32 workers) are captured
  *     as three branches when the workspace has room: the forward beside the backward, and the
  *     aggregation's merge order (which needs the workers' id lists, not their gradients) beside
  *     the backward's sums.  No kernel fills the device there, so the step time is the length of

@@ -176,13 +176,19 @@ struct FusedUpdate {
   void* table; int dtype; int opt; OptParams p; float* state0; float* state1; float* agg_out;
 };
 
-// Rows a lane group has in flight and CTAs per SM.  Measured on B200 (100M x 64 bf16 table, 16
-// workers, 16.7 M contributions to 9.2 M rows): 1 row at 6 CTAs 3.08 ms; 1 row at 4-5 CTAs
-// 3.2-3.4 ms; 2 rows 3.5-4.1 ms; 4 rows 5.0 ms.
+// Rows a lane group has in flight, CTAs per SM and the grid.  The kernel is a chain of dependent
+// loads per row (slots -> positions -> gradient rows), so warps in flight count for more than
+// loads in flight per warp, and the grid decides how close in time neighbouring rows are worked
+// on.  Measured on B200 (100M x 64 bf16 table, Adagrad, 16 workers, 16.7 M contributions to 9.2 M
+// rows; the two separate kernels take 2.73 ms): 1 row, 8 CTAs/SM, grid of 16 resident waves
+// 2.58 ms; 32 waves 2.58; 8 waves 2.62; 4 waves 2.74; 2 waves 2.88; 1 wave 2.95; one row per
+// lane group and no stride 3.30; 6 CTAs/SM 3.05; 2 rows in flight 3.5-4.1; 4 rows 5.0.  Adam
+// needs more registers than 8 CTAs/SM leave and stays at 6.
 constexpr int kFusedRows = 1;
-constexpr int kFusedCtas = 6;
+constexpr int kFusedWaves = 16;
+template <bool ADAM> constexpr int fused_ctas() { return ADAM ? 6 : 8; }
 template <int G, int VPL, bool ADAM, bool BF16>
-__global__ void __launch_bounds__(256, (VPL == 1 ? kFusedCtas : 1))
+__global__ void __launch_bounds__(256, (VPL == 1 ? fused_ctas<ADAM>() : 1))
 agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __restrict__ src,
                   const int32_t* __restrict__ agg_ids, const int64_t* __restrict__ n_agg_dev,
                   int64_t out_cap, const int64_t* __restrict__ n_entries,
@@ -291,10 +297,10 @@ void launch_agg_update(const FusedUpdate& fu, const uint32_t* row_start, const u
                        const int64_t* wuo, const float* weights, int K, cudaStream_t s) {
   const int64_t gpb = 256 / G;
   const int64_t want = (out_cap + gpb - 1) / gpb;
-  const int64_t cap = (int64_t)kNumSM * 16;
-  const unsigned grid = (unsigned)(want > cap ? cap : (want < 1 ? 1 : want));
   const size_t smem = 8 * ((size_t)K + 1) + 4 * (size_t)K;
   const bool adam = fu.opt == ANTDT_OPT_ADAM, bf16 = fu.dtype == ANTDT_BF16;
+  const int64_t cap = (int64_t)kNumSM * (adam ? fused_ctas<true>() : fused_ctas<false>()) * kFusedWaves;
+  const unsigned grid = (unsigned)(want > cap ? cap : (want < 1 ? 1 : want));
 #define FU_GO(A, B)                                                                              \
   ANTDT_LAUNCH("agg_update", (agg_update_kernel<G, VPL, A, B>), grid, 256, smem, s, row_start, src, \
                sp->agg_ids, sp->n_agg, out_cap, n_entries, sp->uniq_grads, sp->in_cap, wuo, weights, K, \
@@ -508,12 +514,13 @@ extern "C" int32_t antdt_weighted_aggregate_backup(const antdt_sparse_part* sp,
 
 // Aggregation followed by the sparse update in one call; with up to 32 workers in one pass over
 // the aggregated rows (agg_update_kernel), otherwise the two steps one after the other.
-extern "C" int32_t antdt_aggregate_update(const antdt_sparse_part* sp, const antdt_dense_part* dp,
-                                          const int64_t* batch_sizes, int32_t n_workers, void* table,
-                                          int32_t dtype, int32_t opt, float lr, float eps, float beta1,
-                                          float beta2, int64_t step, float* state0, float* state1,
-                                          void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
-  using namespace antdt;
+namespace antdt {
+int32_t aggregate_update_forked(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                const int64_t* batch_sizes, int32_t n_workers, void* table,
+                                int32_t dtype, int32_t opt, float lr, float eps, float beta1,
+                                float beta2, int64_t step, float* state0, float* state1, void* ws,
+                                size_t ws_bytes, int32_t* dev_status, void* stream,
+                                const OrderFork* fork) {
   if (!sp || !table || !state0 || step < 1) return ANTDT_ERR_INVALID_ARG;
   if (dtype != ANTDT_F32 && dtype != ANTDT_BF16) return ANTDT_ERR_INVALID_ARG;
   if (sp->dim % (dtype == ANTDT_BF16 ? 8 : 4)) return ANTDT_ERR_INVALID_ARG;
@@ -534,5 +541,17 @@ extern "C" int32_t antdt_aggregate_update(const antdt_sparse_part* sp, const ant
   fu.table = table; fu.dtype = dtype; fu.opt = opt; fu.state0 = state0; fu.state1 = state1;
   fu.agg_out = nullptr;
   fu.p = make_opt_params(lr, eps, beta1, beta2, step);
-  return aggregate_impl(sp, dp, batch_sizes, nullptr, n_workers, ws, ws_bytes, dev_status, stream, &fu);
+  return aggregate_impl(sp, dp, batch_sizes, nullptr, n_workers, ws, ws_bytes, dev_status, stream, &fu,
+                        fork);
+}
+}  // namespace antdt
+
+extern "C" int32_t antdt_aggregate_update(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                          const int64_t* batch_sizes, int32_t n_workers, void* table,
+                                          int32_t dtype, int32_t opt, float lr, float eps, float beta1,
+                                          float beta2, int64_t step, float* state0, float* state1,
+                                          void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  return antdt::aggregate_update_forked(sp, dp, batch_sizes, n_workers, table, dtype, opt, lr, eps, beta1,
+                                        beta2, step, state0, state1, ws, ws_bytes, dev_status, stream,
+                                        nullptr);
 }

@@ -68,6 +68,12 @@ int32_t weighted_aggregate_forked(const antdt_sparse_part* sp, const antdt_dense
                                   const int64_t* batch_sizes, int32_t n_workers, void* ws,
                                   size_t ws_bytes, int32_t* dev_status, void* stream,
                                   const OrderFork* fork);  // aggregate.cu
+int32_t aggregate_update_forked(const antdt_sparse_part* sp, const antdt_dense_part* dp,
+                                const int64_t* batch_sizes, int32_t n_workers, void* table,
+                                int32_t dtype, int32_t opt, float lr, float eps, float beta1,
+                                float beta2, int64_t step, float* state0, float* state1, void* ws,
+                                size_t ws_bytes, int32_t* dev_status, void* stream,
+                                const OrderFork* fork);  // aggregate.cu
 
 int32_t fwd_impl(const void* table, int32_t dtype, int64_t n_rows, int32_t dim, const int32_t* row_ids,
                  int64_t nnz, const int64_t* bag_offsets, int64_t n_bags, float* pooled,

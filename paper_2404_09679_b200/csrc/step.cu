@@ -14,9 +14,10 @@ static int32_t server_step(const antdt_step_desc* d, antdt_sparse_part* sp, cons
                            void* stream, const OrderFork* fork = nullptr, size_t ws_skip = 0) {
   if (d->fuse_update && (d->opt == ANTDT_OPT_ADAGRAD || d->opt == ANTDT_OPT_ADAM)) {
     if (d->n_workers <= kRangeMaxWorkers) sp->agg_grads = nullptr;  // not materialised
-    return antdt_aggregate_update(sp, dp, d->batch_sizes, d->n_workers, d->table, d->dtype, d->opt,
-                                  d->lr, d->eps, d->beta1, d->beta2, d->step, d->state0, d->state1,
-                                  d->ws, d->ws_bytes, d->d_status, stream);
+    return aggregate_update_forked(sp, dp, d->batch_sizes, d->n_workers, d->table, d->dtype, d->opt,
+                                   d->lr, d->eps, d->beta1, d->beta2, d->step, d->state0, d->state1,
+                                   static_cast<char*>(d->ws) + ws_skip, d->ws_bytes - ws_skip,
+                                   d->d_status, stream, fork);
   }
   // a forked step keeps the aggregation's scratch behind the backward's (both are live at once)
   int32_t rc = weighted_aggregate_forked(sp, dp, d->batch_sizes, d->n_workers,
@@ -195,7 +196,7 @@ namespace {
 constexpr int64_t kForkMaxNnz = (int64_t)1 << 22;
 
 size_t fork_ws_skip(const antdt_step_desc* d) {  // 0: no room (or no reason) to fork
-  if (d->nnz < 1 || d->nnz > kForkMaxNnz || d->fuse_update || d->n_workers > antdt::kRangeMaxWorkers ||
+  if (d->nnz < 1 || d->nnz > kForkMaxNnz || d->n_workers > antdt::kRangeMaxWorkers ||
       d->uniq_cap < 1)
     return 0;
   const size_t b = antdt_embbag_bwd_dedup_workspace_bytes(d->nnz, d->n_bags, d->dim, d->n_workers);

@@ -33,13 +33,13 @@ CASES = {
 class _Side:
     """One copy of the model state and buffers, stepped through one of the two entry points."""
 
-    def __init__(self, w, table0, max_nnz, max_bags, graph):
+    def __init__(self, w, table0, max_nnz, max_bags, graph, fuse_update=False):
         self.table = table0.clone()
         self.s0 = torch.zeros(w.V, w.D, device="cuda")
         self.s1 = torch.zeros(w.V, w.D, device="cuda") if w.opt == "adam" else None
         self.buf = StepBuffers(w.D, w.K, max_nnz, max_bags, w.dense_n)
         oc = OptConfig(B.OPTS[w.opt], w.lr, w.eps, w.beta1, w.beta2)
-        self.step = DeviceStep(self.buf, self.table, self.s0, self.s1, oc, w.K)
+        self.step = DeviceStep(self.buf, self.table, self.s0, self.s1, oc, w.K, fuse_update=fuse_update)
         self.graph = graph
 
     def run(self, t, b, F):
@@ -105,6 +105,46 @@ def test_graph_step_equals_plain_step(name):
             G.close(g.agg_grads[:na].cpu().numpy(), want["agg"], rtol=3e-5, atol=2e-6)
     # a replayed or freshly captured graph accounts for the same kernels as the plain launches
     assert all(a == b and a > 0 for a, b in launches), launches
+    B.antdt_bsp_step_graph_reset()
+
+
+@pytest.mark.parametrize("name", ["c1_varying_sizes", "c2_replay"])
+def test_one_pass_server_step_as_graph_equals_plain_and_agrees_with_the_two_kernel_step(name):
+    """fuse_update: aggregation and update in one kernel.  As a graph (three branches on these
+    sizes) it must equal its plain launches bit for bit; against the two-kernel step the table and
+    the accumulator agree to rounding (the weighted sum is formed with fused multiply-adds in the
+    one-pass kernel), step after step on free-running state."""
+    w, n_steps, n_batches = CASES[name]
+    n_steps = min(n_steps, 6)
+    plans = plan_steps(w, n_batches)
+    bm = synth.BatchMaker(w, "cuda")
+    table0 = bm.table()
+    batches = [make_batch(bm, plans[j], j) for j in range(n_batches)]
+    max_nnz = max(b["row_ids"].numel() for b in batches)
+    max_bags = max(b["bag_offsets"].numel() - 1 for b in batches)
+    two = _Side(w, table0, max_nnz, max_bags, graph=False)
+    plain = _Side(w, table0, max_nnz, max_bags, graph=False, fuse_update=True)
+    graph = _Side(w, table0, max_nnz, max_bags, graph=True, fuse_update=True)
+    B.antdt_bsp_step_graph_reset()
+    for s in range(n_steps):
+        b = batches[s % n_batches]
+        n_bags = b["bag_offsets"].numel() - 1
+        for side in (two, plain, graph):
+            side.run(s + 1, b, w.F)
+        torch.cuda.synchronize()
+        for side in (two, plain, graph):
+            assert B.antdt_read_status(side.buf.status) == 0
+        _same(plain.buf.pooled[:n_bags], graph.buf.pooled[:n_bags], f"pooled, step {s}")
+        _same(plain.buf.n_agg, graph.buf.n_agg, f"n_agg, step {s}")
+        na = int(plain.buf.n_agg.item())
+        _same(plain.buf.agg_ids[:na], graph.buf.agg_ids[:na], f"agg_ids, step {s}")
+        _same(plain.table, graph.table, f"table, step {s}")
+        _same(plain.s0, graph.s0, f"state0, step {s}")
+        _same(two.buf.agg_ids[:na], plain.buf.agg_ids[:na], f"agg_ids vs two-kernel step, step {s}")
+        rows = plain.buf.agg_ids[:na].long()
+        G.close_mostly(plain.table[rows].cpu().numpy(), two.table[rows].cpu().numpy(), 5e-5, 2e-6, 1e-3, 2 * w.lr)
+        G.close_mostly(plain.s0[rows].cpu().numpy(), two.s0[rows].cpu().numpy(), 1e-4, 1e-7, 1e-3,
+                       1e-6 + 1e-4 * float(two.s0.abs().max().item()))
     B.antdt_bsp_step_graph_reset()
 
 
