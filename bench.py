@@ -397,8 +397,8 @@ def run_ours(args):
     if world > 1:
         w = w.scaled(seed=w.seed + 1000 * rank)           # independent replicas
     W, K_steps = args.warmup, args.steps
-    # one-pass server step where it measures faster (Adagrad: configs 1, 2, 4), two kernels for Adam
-    args.fuse_update = args.fuse_update or (w.opt == "adagrad" and not args.no_fuse_update)
+    # the one-pass server step measures faster on all five configs; it needs at most 32 workers
+    args.fuse_update = args.fuse_update or (w.K <= 32 and not args.no_fuse_update)
     n_batches = min(3, W + K_steps)
     plans = plan_all(w, max(n_batches, 1))
     bm = synth.BatchMaker(w, dev)
@@ -827,7 +827,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--fuse-update", action="store_true",
                     help="server step through antdt_aggregate_update (aggregated gradients not "
-                         "materialised); the default for the Adagrad configurations, where it is faster")
+                         "materialised); the default")
     ap.add_argument("--no-fuse-update", action="store_true",
                     help="server step as antdt_weighted_aggregate + antdt_sparse_opt_update on every config")
     ap.add_argument("--no-l2-probe", action="store_true",

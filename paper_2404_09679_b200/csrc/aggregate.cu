@@ -180,15 +180,16 @@ struct FusedUpdate {
 // loads per row (slots -> positions -> gradient rows), so warps in flight count for more than
 // loads in flight per warp, and the grid decides how close in time neighbouring rows are worked
 // on.  Measured on B200 (100M x 64 bf16 table, Adagrad, 16 workers, 16.7 M contributions to 9.2 M
-// rows; the two separate kernels take 2.73 ms): 1 row, 8 CTAs/SM, grid of 16 resident waves
-// 2.58 ms; 32 waves 2.58; 8 waves 2.62; 4 waves 2.74; 2 waves 2.88; 1 wave 2.95; one row per
-// lane group and no stride 3.30; 6 CTAs/SM 3.05; 2 rows in flight 3.5-4.1; 4 rows 5.0.  Adam
-// needs more registers than 8 CTAs/SM leave and stays at 6.
+// rows; the two separate kernels take 2.73 ms): 1 row, 8 CTAs/SM, grid of 16 resident waves,
+// parameters and state requested after the sum 2.42 ms (requested before it 2.58); 32 waves 2.58;
+// 8 waves 2.62; 4 waves 2.74; 2 waves 2.88; 1 wave 2.95; one row per lane group and no stride
+// 3.30; 6 CTAs/SM 3.05; 2 rows in flight 3.5-4.1; 4 rows 5.0.  Adam (fp32 rows, 16 and 32
+// workers): 3.10 / 2.13 ms against 3.22 / 2.20 for the two kernels; at 6 CTAs/SM 3.26 / 2.30.
 constexpr int kFusedRows = 1;
 constexpr int kFusedWaves = 16;
-template <bool ADAM> constexpr int fused_ctas() { return ADAM ? 6 : 8; }
+constexpr int kFusedCtas = 8;
 template <int G, int VPL, bool ADAM, bool BF16>
-__global__ void __launch_bounds__(256, (VPL == 1 ? fused_ctas<ADAM>() : 1))
+__global__ void __launch_bounds__(256, (VPL == 1 ? kFusedCtas : 1))
 agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __restrict__ src,
                   const int32_t* __restrict__ agg_ids, const int64_t* __restrict__ n_agg_dev,
                   int64_t out_cap, const int64_t* __restrict__ n_entries,
@@ -237,11 +238,6 @@ agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __rest
       for (int r = 0; r < R; ++r) {
         at[r] = (size_t)(ok[r] ? row[r] : 0) * dim + 4 * (size_t)vi;
         g[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ok[r]) {
-          w[r] = load_row4(table, BF16, at[r]);
-          a0[r] = *reinterpret_cast<const float4*>(state0 + at[r]);
-          if (ADAM) a1[r] = *reinterpret_cast<const float4*>(state1 + at[r]);
-        }
       }
       for (uint32_t e = 0; e < longest; e += 2) {
         float4 v[R][2];
@@ -272,6 +268,16 @@ agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __rest
           }
         }
       }
+      // the row's parameters and state are requested only now: asking for them before the sum
+      // (to overlap their latency with it) costs registers that the 64 warps per SM do not have
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (ok[r]) {
+          w[r] = load_row4(table, BF16, at[r]);
+          a0[r] = *reinterpret_cast<const float4*>(state0 + at[r]);
+          if (ADAM) a1[r] = *reinterpret_cast<const float4*>(state1 + at[r]);
+        }
+      }
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         if (!ok[r]) continue;
@@ -299,7 +305,7 @@ void launch_agg_update(const FusedUpdate& fu, const uint32_t* row_start, const u
   const int64_t want = (out_cap + gpb - 1) / gpb;
   const size_t smem = 8 * ((size_t)K + 1) + 4 * (size_t)K;
   const bool adam = fu.opt == ANTDT_OPT_ADAM, bf16 = fu.dtype == ANTDT_BF16;
-  const int64_t cap = (int64_t)kNumSM * (adam ? fused_ctas<true>() : fused_ctas<false>()) * kFusedWaves;
+  const int64_t cap = (int64_t)kNumSM * kFusedCtas * kFusedWaves;
   const unsigned grid = (unsigned)(want > cap ? cap : (want < 1 ? 1 : want));
 #define FU_GO(A, B)                                                                              \
   ANTDT_LAUNCH("agg_update", (agg_update_kernel<G, VPL, A, B>), grid, 256, smem, s, row_start, src, \
