@@ -181,10 +181,14 @@ struct FusedUpdate {
 // loads in flight per warp, and the grid decides how close in time neighbouring rows are worked
 // on.  Measured on B200 (100M x 64 bf16 table, Adagrad, 16 workers, 16.7 M contributions to 9.2 M
 // rows; the two separate kernels take 2.73 ms): 1 row, 8 CTAs/SM, grid of 16 resident waves,
-// parameters and state requested after the sum 2.42 ms (requested before it 2.58); 32 waves 2.58;
+// parameters and state prefetched towards L2 before the sum and loaded after it 2.33 ms (loaded
+// after it without the prefetch 2.42, loaded before it 2.58); 32 waves 2.58;
 // 8 waves 2.62; 4 waves 2.74; 2 waves 2.88; 1 wave 2.95; one row per lane group and no stride
 // 3.30; 6 CTAs/SM 3.05; 2 rows in flight 3.5-4.1; 4 rows 5.0.  Adam (fp32 rows, 16 and 32
-// workers): 3.10 / 2.13 ms against 3.22 / 2.20 for the two kernels; at 6 CTAs/SM 3.26 / 2.30.
+// workers): 2.91 / 1.96 ms against 3.22 / 2.20 for the two kernels; at 6 CTAs/SM 3.26 / 2.30.
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
 constexpr int kFusedRows = 1;
 constexpr int kFusedWaves = 16;
 constexpr int kFusedCtas = 8;
@@ -238,6 +242,11 @@ agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __rest
       for (int r = 0; r < R; ++r) {
         at[r] = (size_t)(ok[r] ? row[r] : 0) * dim + 4 * (size_t)vi;
         g[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ok[r]) {  // towards L2 now (costs no register), into registers after the sum
+          prefetch_l2(static_cast<const char*>(table) + at[r] * (BF16 ? 2 : 4));
+          prefetch_l2(state0 + at[r]);
+          if (ADAM) prefetch_l2(state1 + at[r]);
+        }
       }
       for (uint32_t e = 0; e < longest; e += 2) {
         float4 v[R][2];
