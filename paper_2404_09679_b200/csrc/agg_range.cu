@@ -265,7 +265,7 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
                   uint32_t dropped, const int64_t* __restrict__ base, int32_t* __restrict__ agg_ids,
                   int64_t out_cap, uint32_t* __restrict__ src, uint32_t* head_bits,
                   int32_t* __restrict__ tile_first, int tile_shift, uint32_t* __restrict__ row_start,
-                  int32_t* status) {
+                  uint8_t* __restrict__ src_worker, int32_t* status) {
   extern __shared__ __align__(16) unsigned char ra_smem[];
   const int R = 1 << r_log2;
   const int nW = R / 32;  // presence words: at most 256 = one per thread
@@ -347,6 +347,7 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
                    const int64_t dest = pc.before + (int64_t)(shp.fc16 ? first_c16[t] : first_c[t]) + slot;
                    const int64_t u = u0 + t;
                    src[dest] = (uint32_t)j;
+                   if (src_worker) src_worker[dest] = (uint8_t)w;  // saves the reader a search
                    if (slot == 0 && u < out_cap) {
                      agg_ids[u] = (int32_t)id;
                      if (row_start) row_start[u] = (uint32_t)dest;  // the row's first merge slot
@@ -389,7 +390,8 @@ void range_prepare_device() {
 void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t in_cap, int64_t n_rows,
                        int K, uint32_t dropped_bits, int32_t* agg_ids, int64_t* n_agg, int64_t out_cap,
                        int64_t* wuo_out, int64_t* n_entries, uint32_t* src, uint32_t* head_bits,
-                       int32_t* tile_first, int tile, uint32_t* row_start, const float* weights_host,
+                       int32_t* tile_first, int tile, uint32_t* row_start, uint8_t* src_worker,
+                       const float* weights_host,
                        float* weights_dev, char* ws, const RangeLayout& L, int32_t* status,
                        cudaStream_t s) {
   range_prepare_device();
@@ -415,7 +417,7 @@ void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t i
   cudaMemsetAsync(tile_first, 0, 4 * ((size_t)((in_cap + tile - 1) >> tile_shift) + 1), s);
   ANTDT_LAUNCH("agg_range_emit", range_emit_kernel, (unsigned)P, kRaThreads, emit_smem(r_log2, K), s,
                uniq_ids, bnd, wuo_out, K, P, r_log2, n_rows, dropped_bits, base, agg_ids, out_cap, src,
-               head_bits, tile_first, tile_shift, row_start, status);
+               head_bits, tile_first, tile_shift, row_start, src_worker, status);
 }
 
 }  // namespace antdt

@@ -48,12 +48,14 @@ void range_prepare_device();
 //   head_bits           bit i set iff slot i is the first contribution of its row (zeroed here)
 //   tile_first          index into agg_ids of the row that slot t*tile belongs to
 //   row_start [out_cap] merge slot of the first contribution of each row of agg_ids, or nullptr
+//   src_worker [in_cap] the worker of every merge slot (one byte), or nullptr
 //   weights_host [K]    the workers' weights; the first kernel carries them to weights_dev [K]
 //                       as a parameter (nullptr: the caller has put them there already)
 void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t in_cap, int64_t n_rows,
                        int K, uint32_t dropped_bits, int32_t* agg_ids, int64_t* n_agg, int64_t out_cap,
                        int64_t* wuo_out, int64_t* n_entries, uint32_t* src, uint32_t* head_bits,
-                       int32_t* tile_first, int tile, uint32_t* row_start, const float* weights_host,
+                       int32_t* tile_first, int tile, uint32_t* row_start, uint8_t* src_worker,
+                       const float* weights_host,
                        float* weights_dev, char* ws, const RangeLayout& L, int32_t* status,
                        cudaStream_t s);
 

@@ -23,7 +23,7 @@ struct AggLayout {
   RangeLayout range;
   size_t range_ws;
   size_t sort_ws, bounds, weights, wuo, cwuo, drop, keys_a, keys_b, src, vals_t, run_start, head_bits,
-      tile_first, head_part, tail_part, row_start, bytes;
+      tile_first, head_part, tail_part, row_start, src_worker, bytes;
 };
 
 AggLayout agg_layout(int64_t in_cap, int K, int dim) {
@@ -49,6 +49,7 @@ AggLayout agg_layout(int64_t in_cap, int K, int dim) {
   L.head_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
   L.tail_part = o;  o = align_up(o + 4 * n_tiles * (size_t)dim);
   L.row_start = o;  o = align_up(o + 4 * (n + 1));
+  L.src_worker = o; o = align_up(o + n + 1);
   L.range_ws = o;
   if (K <= kRangeMaxWorkers) {  // scratch of the range-partitioned merge (up to 32 workers)
     L.range = range_layout(K);
@@ -197,12 +198,11 @@ __global__ void __launch_bounds__(256, (VPL == 1 ? kFusedCtas : 1))
 agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __restrict__ src,
                   const int32_t* __restrict__ agg_ids, const int64_t* __restrict__ n_agg_dev,
                   int64_t out_cap, const int64_t* __restrict__ n_entries,
-                  const float* __restrict__ grads, int64_t in_cap, const int64_t* __restrict__ wuo,
-                  const float* __restrict__ weights, int K, void* table, int64_t n_rows, int dim,
-                  OptParams p, float* state0, float* state1, float* __restrict__ agg_out) {
-  extern __shared__ int64_t s_wu[];  // wuo [K+1], then K weights
-  float* s_w = reinterpret_cast<float*>(s_wu + (K + 1));
-  for (int i = threadIdx.x; i <= K; i += blockDim.x) s_wu[i] = wuo[i];
+                  const float* __restrict__ grads, int64_t in_cap,
+                  const uint8_t* __restrict__ src_worker, const float* __restrict__ weights, int K,
+                  void* table, int64_t n_rows, int dim, OptParams p, float* state0, float* state1,
+                  float* __restrict__ agg_out) {
+  extern __shared__ float s_w[];  // the K weights
   for (int i = threadIdx.x; i < K; i += blockDim.x) s_w[i] = weights[i];
   __syncthreads();
   constexpr int R = VPL == 1 ? kFusedRows : 1;  // rows a lane group has in flight
@@ -261,7 +261,7 @@ agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __rest
             if (o < s1[r]) {
               const uint32_t pos = __ldg(src + o);
               if ((int64_t)pos < in_cap) {
-                int wl = interval_of(s_wu, K + 1, (int64_t)pos);
+                const int wl = (int)__ldg(src_worker + o);  // written beside src[o] by the merge
                 wt[r][t] = s_w[wl > K - 1 ? K - 1 : wl];
                 v[r][t] = ldg_f4(grads + (size_t)pos * dim + 4 * vi);
               }
@@ -309,16 +309,16 @@ agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __rest
 template <int G, int VPL>
 void launch_agg_update(const FusedUpdate& fu, const uint32_t* row_start, const uint32_t* src,
                        const antdt_sparse_part* sp, int64_t out_cap, const int64_t* n_entries,
-                       const int64_t* wuo, const float* weights, int K, cudaStream_t s) {
+                       const uint8_t* src_worker, const float* weights, int K, cudaStream_t s) {
   const int64_t gpb = 256 / G;
   const int64_t want = (out_cap + gpb - 1) / gpb;
-  const size_t smem = 8 * ((size_t)K + 1) + 4 * (size_t)K;
+  const size_t smem = 4 * (size_t)K;
   const bool adam = fu.opt == ANTDT_OPT_ADAM, bf16 = fu.dtype == ANTDT_BF16;
   const int64_t cap = (int64_t)kNumSM * kFusedCtas * kFusedWaves;
   const unsigned grid = (unsigned)(want > cap ? cap : (want < 1 ? 1 : want));
 #define FU_GO(A, B)                                                                              \
   ANTDT_LAUNCH("agg_update", (agg_update_kernel<G, VPL, A, B>), grid, 256, smem, s, row_start, src, \
-               sp->agg_ids, sp->n_agg, out_cap, n_entries, sp->uniq_grads, sp->in_cap, wuo, weights, K, \
+               sp->agg_ids, sp->n_agg, out_cap, n_entries, sp->uniq_grads, sp->in_cap, src_worker, weights, K, \
                fu.table, sp->n_rows, sp->dim, fu.p, fu.state0, fu.state1, fu.agg_out)
   if (adam) { if (bf16) FU_GO(true, true); else FU_GO(true, false); }
   else      { if (bf16) FU_GO(false, true); else FU_GO(false, false); }
@@ -440,7 +440,8 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
                         sp->agg_ids, sp->n_agg, agg_cap, (int64_t*)(w8 + L.wuo), bounds,
                         (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.head_bits),
                         (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap),
-                        fu ? (uint32_t*)(w8 + L.row_start) : nullptr, hw, (float*)(w8 + L.weights),
+                        fu ? (uint32_t*)(w8 + L.row_start) : nullptr,
+                        fu ? (uint8_t*)(w8 + L.src_worker) : nullptr, hw, (float*)(w8 + L.weights),
                         w8 + L.range_ws, L.range, dev_status, so);
       if (fork && (cudaEventRecord(fork->order_done, so) != cudaSuccess ||
                    cudaStreamWaitEvent(s, fork->order_done, 0) != cudaSuccess))
@@ -454,10 +455,10 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
       f.agg_out = sp->agg_grads;
       const uint32_t* rs = (const uint32_t*)(w8 + L.row_start);
       const uint32_t* src = (const uint32_t*)(w8 + L.src);
-      const int64_t* wuo = (const int64_t*)(w8 + L.wuo);
+      const uint8_t* sw = (const uint8_t*)(w8 + L.src_worker);
       const float* wts = (const float*)(w8 + L.weights);
       const int nvec = sp->dim / 4;
-#define FU_CASE(G, VPL) launch_agg_update<G, VPL>(f, rs, src, sp, agg_cap, bounds, wuo, wts, K, s)
+#define FU_CASE(G, VPL) launch_agg_update<G, VPL>(f, rs, src, sp, agg_cap, bounds, sw, wts, K, s)
       if (nvec <= 1) FU_CASE(1, 1);
       else if (nvec <= 2) FU_CASE(2, 1);
       else if (nvec <= 4) FU_CASE(4, 1);
