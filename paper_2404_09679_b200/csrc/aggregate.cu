@@ -208,25 +208,27 @@ agg_update_kernel(const uint32_t* __restrict__ row_start, const uint32_t* __rest
   constexpr int R = VPL == 1 ? kFusedRows : 1;  // rows a lane group has in flight
   const int lg = threadIdx.x & (G - 1);
   const int nvec = dim / 4;
-  const int64_t n = min(*n_agg_dev, out_cap);
+  // 32-bit row numbers and slots (fewer than 2^31 of each): the kernel is bound by its instruction
+  // stream and by the registers that live across the chain of loads
+  const uint32_t n = (uint32_t)min(*n_agg_dev, out_cap);
   const uint32_t total = (uint32_t)min(n_entries[1], in_cap);
-  const int64_t stride = (int64_t)gridDim.x * (256 / G);
-  for (int64_t u0 = (int64_t)blockIdx.x * (256 / G) + threadIdx.x / G; u0 < n; u0 += R * stride) {
+  const uint32_t stride = gridDim.x * (256 / G);
+  for (uint32_t u0 = blockIdx.x * (256 / G) + threadIdx.x / G; u0 < n; u0 += R * stride) {
     uint32_t s0[R], s1[R];
-    int64_t row[R];
+    int32_t row[R];
     bool ok[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      const int64_t u = u0 + r * stride;
+      const uint32_t u = u0 + r * stride;
       ok[r] = u < n;
       s0[r] = ok[r] ? __ldg(row_start + u) : 0u;
       s1[r] = ok[r] ? (u + 1 < n ? __ldg(row_start + u + 1) : total) : 0u;
-      row[r] = ok[r] ? (int64_t)__ldg(agg_ids + u) : -1;
+      row[r] = ok[r] ? __ldg(agg_ids + u) : -1;
     }
     uint32_t longest = 0;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      ok[r] = ok[r] && row[r] >= 0 && row[r] < n_rows && s0[r] <= total;  // else flagged by the merge
+      ok[r] = ok[r] && (uint32_t)row[r] < (uint32_t)n_rows && s0[r] <= total;  // else flagged by the merge
       if (s1[r] > total) s1[r] = total;
       if (s1[r] > s0[r] + (uint32_t)K) s1[r] = s0[r] + (uint32_t)K;  // a row has at most K contributions
       if (!ok[r]) s1[r] = s0[r];
