@@ -44,6 +44,33 @@ def test_fwd_matches_checker(D, bf16):
     assert np.all(got[np.diff(off) == 0] == 0)
 
 
+@pytest.mark.parametrize("D,bf16", [(64, False), (64, True)])
+def test_fwd_short_bags_over_several_turns(D, bf16):
+    """Short bags (under 8 ids on average) take the kernel whose lane groups stride over the bags
+    with a capped grid; 700 k bags of 16-lane rows are more than one turn for every group.  A few
+    ids out of range are planted: flagged, and they contribute nothing."""
+    rng = np.random.default_rng(7 + bf16)
+    V, n_bags = 4000, 700_001
+    W = rng.normal(0, 0.01, size=(V, D)).astype(np.float32)
+    Wt = _bf16_bits(W) if bf16 else W
+    ids, off = random_bags(rng, n_bags, V, 6)                # 0..6 ids per bag, empties included
+    got, code = G.gpu_fwd(Wt, ids, off)
+    assert code == 0
+    want = oracle.embbag_fwd(Wt, ids, off)
+    G.close(got, want)
+    assert np.all(got[np.diff(off) == 0] == 0)
+    bad = ids.copy()
+    where = rng.choice(len(ids), size=50, replace=False)
+    bad[where] = V + 3
+    got2, code = G.gpu_fwd(Wt, bad, off)
+    assert code == B.ERR_ID_OUT_OF_RANGE
+    keep = np.ones(len(ids), bool)
+    keep[where] = False
+    off2 = np.concatenate([[0], np.cumsum(np.add.reduceat(keep, off[:-1].clip(max=len(ids) - 1)) *
+                                          (np.diff(off) > 0))]).astype(np.int64)
+    G.close(got2, oracle.embbag_fwd(Wt, ids[keep], off2))
+
+
 def test_fwd_one_hot_is_bit_exact_and_empty_input_is_fine():
     rng = np.random.default_rng(1)
     V, D, n = 1000, 32, 777
