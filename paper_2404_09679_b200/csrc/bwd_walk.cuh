@@ -45,6 +45,7 @@ struct WalkScratch {
   float* tail_part;   // [n_stretches, dim]
   uint8_t* flags;     // [n_stretches]
   int32_t* tasks;     // [2 n_stretches + 4]
+  bool tasks_zeroed = false;  // the caller has cleared the list's counter on this stream already
 };
 inline int walk_tiles_per_stretch(int dim) {  // = lane groups per CTA, see launch_bwd_walk
   const int nvec = dim / 4;
@@ -366,7 +367,7 @@ void launch_bwd_walk_t(const TileArgs& a_in, const WalkScratch& ws, const char* 
     }
   }
   if (a.walk && a.tile_end > a.tile_begin) {
-    if (a.tile_begin == 0) cudaMemsetAsync(ws.tasks, 0, 8, s);  // a new list
+    if (a.tile_begin == 0 && !ws.tasks_zeroed) cudaMemsetAsync(ws.tasks, 0, 8, s);  // a new list
     const unsigned grid = (unsigned)((a.tile_end - a.tile_begin + TPS - 1) / TPS);
     const int vec = aligned16(a.payload) ? 1 : 0;
     ANTDT_LAUNCH(name_tiles, (bwd_walk_kernel<G, VPL, TILE>), grid, kRedThreads, smem, s, a, a.payload,

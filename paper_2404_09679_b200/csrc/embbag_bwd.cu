@@ -70,7 +70,14 @@ bwd_prep_kernel(const int64_t* __restrict__ wso, int K, int F, const int64_t* __
 // occurrence of the warp's range finds its bag by a 5-step search over the lanes' values.
 __global__ void __launch_bounds__(256)
 expand_bags_kernel(const int64_t* __restrict__ bag_offsets, int64_t n_bags, int64_t nnz,
-                   uint32_t* __restrict__ occ_bag, int32_t* status) {
+                   uint32_t* __restrict__ occ_bag, int32_t* status, uint32_t* __restrict__ zero_words,
+                   int64_t n_zero_words, int32_t* __restrict__ zero_pair) {
+  // scratch that later kernels of the call expect zeroed (the run heads' bit mask, the fix-up's
+  // task counter): cleared here, on the way, instead of by two memsets in the chain of launches
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_zero_words;
+       i += (int64_t)gridDim.x * blockDim.x)
+    zero_words[i] = 0u;
+  if (blockIdx.x == 0 && threadIdx.x < 2 && zero_pair) zero_pair[threadIdx.x] = 0;
   const int lane = threadIdx.x & 31;
   const int64_t b0 = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32;
   if (b0 >= n_bags) return;
@@ -176,16 +183,19 @@ int32_t bwd_dedup_impl(
   // payload ping-pong ends in sorted_occ: start in whichever buffer makes the last pass land there
   uint32_t* occ_out = reinterpret_cast<uint32_t*>(sorted_occ);
   uint32_t* expand_to = (P % 2 == 1) ? vals_t : occ_out;
+  bool scratch_zeroed = false;
   if (n_bags > 0 && nnz > 0) {
     const unsigned grid = (unsigned)((n_bags + 32 * 8 - 1) / (32 * 8));
     ANTDT_LAUNCH("expand_bags", expand_bags_kernel, grid, 256, 0, s, bag_offsets, n_bags, nnz,
-                 expand_to, dev_status);
+                 expand_to, dev_status, (uint32_t*)(w8 + L.head_bits), (int64_t)head_bits_words(nnz),
+                 (int32_t*)(w8 + L.tasks));
+    scratch_zeroed = true;
   }
   segsort_run(reinterpret_cast<const uint32_t*>(row_ids), expand_to, keys_a, occ_out, keys_b,
               vals_t, key_bits, n_rows, nnz, sort_ws, L.sort, dev_status, s);
   segsort_runs(keys_a, nnz, uniq_ids, seg_offsets, worker_uniq_offsets, nullptr, out_cap,
                (uint32_t*)(w8 + L.head_bits), (int32_t*)(w8 + L.tile_first), tile_len, sort_ws,
-               L.sort, dev_status, s);
+               L.sort, dev_status, s, false, scratch_zeroed);
   if (ids_done && cudaEventRecord(ids_done, s) != cudaSuccess) return ANTDT_ERR_CUDA;
   if (nnz > 0) {
     TileArgs t;
@@ -208,6 +218,7 @@ int32_t bwd_dedup_impl(
     tasks.tail_part = (float*)(w8 + L.tail_part);
     tasks.flags = (uint8_t*)(w8 + L.flags);
     tasks.tasks = (int32_t*)(w8 + L.tasks);
+    tasks.tasks_zeroed = scratch_zeroed;
     if (!arrival || arrival->n < 1) {
       launch_bwd_walk(t, tasks, "seg_reduce_tiles", "seg_reduce_fixup", s);
     } else {

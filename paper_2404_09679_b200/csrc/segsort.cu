@@ -719,7 +719,7 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
 void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys,
                   int64_t* run_start, int64_t* seg_runs, int64_t* n_runs_out, int64_t out_cap,
                   uint32_t* head_bits, int32_t* tile_first, int tile, char* ws,
-                  const SortLayout& L, int32_t* status, cudaStream_t s, bool agg) {
+                  const SortLayout& L, int32_t* status, cudaStream_t s, bool agg, bool head_bits_zeroed) {
   const SortDesc* desc = (const SortDesc*)(ws + L.desc);
   const int64_t* seg_bounds = (const int64_t*)(ws + L.seg_bounds);
   const int32_t* seg_first = (const int32_t*)(ws + L.seg_first);
@@ -727,7 +727,7 @@ void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys
   const int64_t* chunk_begin = (const int64_t*)(ws + L.chunk_begin);
   const int64_t* chunk_end = (const int64_t*)(ws + L.chunk_end);
   int64_t* chunk_runs = (int64_t*)(ws + L.chunk_runs);
-  if (head_bits) cudaMemsetAsync(head_bits, 0, head_bits_words(n_cap) * 4, s);
+  if (head_bits && !head_bits_zeroed) cudaMemsetAsync(head_bits, 0, head_bits_words(n_cap) * 4, s);
   int tile_shift = 0;
   while ((1 << tile_shift) < tile) ++tile_shift;  // tile is a power of two
   ANTDT_LAUNCH(agg ? "agg_runs_count" : "runs_count", runs_count_kernel, L.max_chunks, kRunThreads, 0, s, sorted_keys,

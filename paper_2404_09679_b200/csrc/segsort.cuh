@@ -92,12 +92,13 @@ void segsort_run(const uint32_t* keys_in, const uint32_t* vals_in, uint32_t* key
 //   run_start  [out_cap+1]  first element of each run; entry [n_runs] = n
 //   seg_runs   [S+1]        runs before each segment; [S] = n_runs  (may be nullptr)
 //   n_runs_out one int64    (may be nullptr)
-//   head_bits  [head_bits_words(n_cap)] bit i set iff element i starts a run (zeroed here)
+//   head_bits  [head_bits_words(n_cap)] bit i set iff element i starts a run (zeroed here unless head_bits_zeroed)
 //   tile_first [n_cap/tile+1] run index of element t*tile (may be nullptr); tile a power of 2
 // More runs than out_cap -> CAPACITY in status, the excess is not written.
 void segsort_runs(const uint32_t* sorted_keys, int64_t n_cap, int32_t* uniq_keys,
                   int64_t* run_start, int64_t* seg_runs, int64_t* n_runs_out, int64_t out_cap,
                   uint32_t* head_bits, int32_t* tile_first, int tile, char* ws,
-                  const SortLayout& L, int32_t* status, cudaStream_t s, bool agg = false);
+                  const SortLayout& L, int32_t* status, cudaStream_t s, bool agg = false,
+                  bool head_bits_zeroed = false);  // true: the caller cleared head_bits on this stream
 
 }  // namespace antdt
