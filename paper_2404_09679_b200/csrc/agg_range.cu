@@ -298,7 +298,8 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
   // hb word i is global head-bit word (before >> 5) + i, same bit positions
   const int hb_shift = (int)(pc.before & 31);
   const int n_hw = (hb_shift + pc.entries + 31) >> 5;
-  for (int i = tid; i < n_hw; i += kRaThreads) hb[i] = 0u;
+  if (head_bits)  // (a reader that goes by row_start needs neither the head bits nor tile_first)
+    for (int i = tid; i < n_hw; i += kRaThreads) hb[i] = 0u;
   if (tid < nW) pres[tid] = 0u;
   {
     uint4* m4 = reinterpret_cast<uint4*>(mask);
@@ -325,14 +326,14 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
     for (uint32_t rest = pw; rest; rest &= rest - 1u) {
       if (shp.fc16) first_c16[t++] = (unsigned short)first;
       else first_c[t++] = (uint32_t)first;
-      atomicOr(&hb[(hb_shift + first) >> 5], 1u << ((hb_shift + first) & 31));
+      if (head_bits) atomicOr(&hb[(hb_shift + first) >> 5], 1u << ((hb_shift + first) & 31));
       first += __popc(workers_of(tid * 32 + __ffs((int)rest) - 1));
     }
   }
   __syncthreads();
 
   // whole words of the head-bit mask are stored, words shared with a neighbour range are merged
-  for (int i = tid; i < n_hw; i += kRaThreads) {
+  for (int i = tid; head_bits && i < n_hw; i += kRaThreads) {
     const uint32_t word = hb[i];
     if (word == 0u) continue;
     const int64_t g = (pc.before >> 5) + i;
@@ -352,7 +353,7 @@ range_emit_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ b
                      agg_ids[u] = (int32_t)id;
                      if (row_start) row_start[u] = (uint32_t)dest;  // the row's first merge slot
                    }
-                   if ((dest & tile_mask) == 0) tile_first[dest >> tile_shift] = (int32_t)u;
+                   if (tile_first && (dest & tile_mask) == 0) tile_first[dest >> tile_shift] = (int32_t)u;
                  });
 }
 
@@ -412,9 +413,9 @@ void range_merge_order(const int32_t* uniq_ids, const int64_t* wuo_in, int64_t i
                uniq_ids, bnd, wuo_out, K, P, r_log2, n_rows, dropped_bits, distinct, status);
   ANTDT_LAUNCH("agg_range_scan", range_scan_kernel, 1, 1024, 0, s, distinct, P, base, n_agg, out_cap,
                status);
-  cudaMemsetAsync(head_bits, 0, head_bits_words(in_cap) * 4, s);
+  if (head_bits) cudaMemsetAsync(head_bits, 0, head_bits_words(in_cap) * 4, s);
   // every tile's entry is written unless ids were skipped as invalid: start from a valid index
-  cudaMemsetAsync(tile_first, 0, 4 * ((size_t)((in_cap + tile - 1) >> tile_shift) + 1), s);
+  if (tile_first) cudaMemsetAsync(tile_first, 0, 4 * ((size_t)((in_cap + tile - 1) >> tile_shift) + 1), s);
   ANTDT_LAUNCH("agg_range_emit", range_emit_kernel, (unsigned)P, kRaThreads, emit_smem(r_log2, K), s,
                uniq_ids, bnd, wuo_out, K, P, r_log2, n_rows, dropped_bits, base, agg_ids, out_cap, src,
                head_bits, tile_first, tile_shift, row_start, src_worker, status);

@@ -47,6 +47,8 @@ void range_prepare_device();
 //                       slots ordered by (row id, worker)
 //   head_bits           bit i set iff slot i is the first contribution of its row (zeroed here)
 //   tile_first          index into agg_ids of the row that slot t*tile belongs to
+//                       (head_bits and tile_first may both be nullptr: a reader that goes by
+//                       row_start needs neither)
 //   row_start [out_cap] merge slot of the first contribution of each row of agg_ids, or nullptr
 //   src_worker [in_cap] the worker of every merge slot (one byte), or nullptr
 //   weights_host [K]    the workers' weights; the first kernel carries them to weights_dev [K]

@@ -440,8 +440,8 @@ int32_t aggregate_impl(const antdt_sparse_part* sp, const antdt_dense_part* dp,
       if (fork && cudaStreamWaitEvent(so, fork->ids_ready, 0) != cudaSuccess) return ANTDT_ERR_CUDA;
       range_merge_order(sp->uniq_ids, sp->worker_uniq_offsets, in_cap, sp->n_rows, K, dropped_bits,
                         sp->agg_ids, sp->n_agg, agg_cap, (int64_t*)(w8 + L.wuo), bounds,
-                        (uint32_t*)(w8 + L.src), (uint32_t*)(w8 + L.head_bits),
-                        (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap),
+                        (uint32_t*)(w8 + L.src), fu ? nullptr : (uint32_t*)(w8 + L.head_bits),
+                        fu ? nullptr : (int32_t*)(w8 + L.tile_first), red_tile_for(in_cap),
                         fu ? (uint32_t*)(w8 + L.row_start) : nullptr,
                         fu ? (uint8_t*)(w8 + L.src_worker) : nullptr, hw, (float*)(w8 + L.weights),
                         w8 + L.range_ws, L.range, dev_status, so);
