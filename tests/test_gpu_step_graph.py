@@ -25,6 +25,8 @@ CASES = {
     "c1_varying_sizes": (synth.WORKLOADS[1], 12, 12),
     # fixed sizes, two batches in rotation: every step after the first two is a replay
     "c2_replay": (synth.WORKLOADS[2].scaled(V=26 * 50_000), 8, 2),
+    # Adagrad with a dense part: the three-branch graph with the dense weighted sum behind the join
+    "c1_dense_adagrad": (synth.WORKLOADS[1].scaled(dense_n=8192), 6, 3),
     # Adam + dense part: issued as plain launches by the entry point
     "c3_adam_dense": (synth.WORKLOADS[3].scaled(B=2048, V=200_000, dense_n=65_536), 10, 3),
 }
@@ -108,7 +110,7 @@ def test_graph_step_equals_plain_step(name):
     B.antdt_bsp_step_graph_reset()
 
 
-@pytest.mark.parametrize("name", ["c1_varying_sizes", "c2_replay"])
+@pytest.mark.parametrize("name", ["c1_varying_sizes", "c2_replay", "c1_dense_adagrad"])
 def test_one_pass_server_step_as_graph_equals_plain_and_agrees_with_the_two_kernel_step(name):
     """fuse_update: aggregation and update in one kernel.  As a graph (three branches on these
     sizes) it must equal its plain launches bit for bit; against the two-kernel step the table and
@@ -140,6 +142,9 @@ def test_one_pass_server_step_as_graph_equals_plain_and_agrees_with_the_two_kern
         _same(plain.buf.agg_ids[:na], graph.buf.agg_ids[:na], f"agg_ids, step {s}")
         _same(plain.table, graph.table, f"table, step {s}")
         _same(plain.s0, graph.s0, f"state0, step {s}")
+        if w.dense_n:
+            _same(plain.buf.dense_out, graph.buf.dense_out, f"dense_out, step {s}")
+            _same(two.buf.dense_out, plain.buf.dense_out, f"dense_out vs two-kernel step, step {s}")
         _same(two.buf.agg_ids[:na], plain.buf.agg_ids[:na], f"agg_ids vs two-kernel step, step {s}")
         rows = plain.buf.agg_ids[:na].long()
         G.close_mostly(plain.table[rows].cpu().numpy(), two.table[rows].cpu().numpy(), 5e-5, 2e-6, 1e-3, 2 * w.lr)
