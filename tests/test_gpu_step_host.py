@@ -124,8 +124,10 @@ def test_single_call_device_step_equals_the_four_calls():
         assert torch.equal(t_b, t_a) and torch.equal(s0_b, s0_a) and torch.equal(s1_b, s1_a)
 
 
-def test_two_host_steps_in_flight_equal_one_at_a_time():
-    """Two staging sets alternated with staging_idle: the copies of a step run under the kernels
+@pytest.mark.parametrize("fuse_update", [False, True])
+def test_two_host_steps_in_flight_equal_one_at_a_time(fuse_update):
+    """(fuse_update: the server step in one pass, as bench.py's end-to-end leg runs it.)
+    Two staging sets alternated with staging_idle: the copies of a step run under the kernels
     of the step before it.  Results (host outputs of every step, table and state at the end) must
     be bit-identical to the same steps issued one at a time."""
     from paper_2404_09679_b200.step import HostStaging, HostStep
@@ -148,7 +150,7 @@ def test_two_host_steps_in_flight_equal_one_at_a_time():
         s0 = torch.zeros(w.V, w.D, device="cuda")
         buf = StepBuffers(w.D, w.K, max_nnz, max_bags, w.dense_n)
         sets = [HostStaging(w.D, w.K, max_nnz, max_bags, w.dense_n) for _ in range(2)]
-        hs = HostStep(buf, table, s0, None, oc, w.K)
+        hs = HostStep(buf, table, s0, None, oc, w.K, fuse_update)
         torch.cuda.synchronize()
         outs, pending = [], None
 
