@@ -48,6 +48,34 @@ def test_lambda_test_flags_a_worker_exactly_at_the_threshold():
     assert t.sum() == 0 and p.sum() == 0 and a == 0
 
 
+def test_persistent_test_compares_with_the_mean_of_the_long_windows():
+    # BPTs of worker 0: 1, 1, 1, 4; of worker 1: 2, 2, 2, 4.  Short window (1 report): 4 and 4, mean 4.
+    # Long window (4 reports): 1.75 and 2.5, mean 2.125.  lambda = 1.1: worker 1 is a persistent
+    # straggler (2.5 >= 1.1 * 2.125 = 2.3375) although nobody is a transient one (4 < 4.4); measured
+    # against the short windows' mean (4.4) it would not be flagged.
+    rep = []
+    for k in range(4):
+        rep += [(0, 32, 4.0 if k == 3 else 1.0), (1, 32, 4.0 if k == 3 else 2.0)]
+    v, t, p, a = oracle.ctl_decide(rep, 2, 1, 4, 1.1)
+    assert t.tolist() == [0, 0] and p.tolist() == [0, 1] and a == 2
+
+
+def test_window_means_divide_by_the_reports_each_worker_has():
+    # worker 1 joined late: two reports of 3 s against worker 0's four of 1 s; long window 4, short
+    # window 1.  Its long-window MEAN is 3 (not 6/4, and not the sum 6): 3 >= 1.4 * mean(1, 3) = 2.8.
+    rep = [(0, 16, 1.0), (0, 16, 1.0), (0, 16, 1.0), (1, 16, 3.0), (0, 16, 1.0), (1, 16, 3.0)]
+    v, t, p, a = oracle.ctl_decide(rep, 2, 1, 4, 1.4)
+    assert p.tolist() == [0, 1] and t.tolist() == [0, 1] and a == 2
+    # with lambda 1.6 the threshold is 3.2: not flagged (a window mean of 6/1 or 6/2 * ... would be)
+    v, t, p, a = oracle.ctl_decide(rep, 2, 1, 4, 1.6)
+    assert p.sum() == 0 and t.sum() == 0 and a == 0
+    # the same for the short window: two reports of 1 s against one report of 1.5 s, window 2:
+    # means 1 and 1.5 (sums would be 2 and 1.5 and flag the wrong worker), threshold 1.1 * 1.25
+    rep = [(0, 16, 1.0), (0, 16, 1.0), (1, 16, 1.5)]
+    v, t, p, a = oracle.ctl_decide(rep, 2, 2, 2, 1.1)
+    assert t.tolist() == [0, 1] and p.tolist() == [0, 1]
+
+
 def test_throughput_is_mean_of_per_report_rates():
     rep = [(0, 100, 1.0), (0, 300, 2.0), (1, 100, 1.0), (1, 100, 1.0)]
     v, _, _, _ = oracle.ctl_decide(rep, 2, 5, 5, 1.5)

@@ -107,6 +107,11 @@ def test_proportional_min_batch_clamp():
     v = [10.0, 10.0, 0.01, 0.01]
     b = oracle.batch_sizes(v, 4, 1000, "proportional", 100)
     assert b.sum() == 1000 and b.tolist() == [400, 400, 100, 100]
+    # what is left after the clamped worker's share goes to the others in proportion to THEIR
+    # speeds: 90 * 3/4 = 67.5 and 90 * 1/4 = 22.5, the odd unit to the lower index.  (Two equal
+    # fast workers would hide a split of the whole batch instead of the remainder: 50 + 50 comes
+    # back to 45 + 45 whichever way the surplus is taken off.)
+    assert oracle.batch_sizes([3.0, 1.0, 0.02], 3, 100, "proportional", 10).tolist() == [68, 22, 10]
     with pytest.raises(oracle.OracleError):
         oracle.batch_sizes(v, 4, 1000, "proportional", 251)
     with pytest.raises(oracle.OracleError):
@@ -206,6 +211,46 @@ def test_drop_on_the_step_that_finishes_a_shard_loses_no_sample():
     assert d.shard_info(0)[0] == 2
     d.requeue_worker(0)
     assert d.shard_info(0)[0] == 2
+
+
+def test_requeue_order_when_a_dropped_worker_finished_two_shards_in_one_step():
+    # 33 samples, B = 10, M = 1: shards 0..2 of 10 samples and the short tail shard 3 = [30, 33).
+    # A worker can only finish two shards in one step when the second is that tail.
+    # Step 1 (speeds 8:1:1 -> batches 8/1/1): worker 0 holds shard 0 (8 used), worker 1 shard 1,
+    # worker 2 shard 2; the queue is [3].  Workers 1 and 2 are dropped: queue [3, 1, 2].
+    # Step 2 (only worker 0 gets samples): it finishes shard 0 (2 samples), takes and finishes the
+    # tail (3 samples) and takes 5 of shard 1; the queue is [2].  Worker 0 is dropped: the shards it
+    # finished in this step come back behind what is queued, the older completion first, then the
+    # one it is DOING (Section V-C.3): [2, 0, 3, 1].
+    d = _mk(33, 10, 1, 3)
+    rc, bsz, ro, rg, cnt = d.plan([8.0, 1.0, 1.0])
+    assert rc == 0 and bsz.tolist() == [8, 1, 1] and rg.tolist() == [[0, 8], [10, 1], [20, 1]]
+    d.requeue_worker(1)
+    d.requeue_worker(2)
+    rc, bsz, ro, rg, cnt = d.plan([1.0, 1e-9, 1e-9])
+    assert rc == 0 and bsz.tolist() == [10, 0, 0]
+    assert rg[ro[0]:ro[1]].tolist() == [[8, 2], [30, 3], [10, 5]]
+    assert d.shard_info(0)[0] == 2 and d.shard_info(3)[0] == 2 and d.shard_info(1)[:2] == (1, 0)
+    d.requeue_worker(0)
+    assert d.counts() == (4, 0, 0)
+    served = []
+    while True:                       # worker 1 alone drains the queue, a whole batch per step
+        rc, bsz, ro, rg, cnt = d.plan([1e-9, 1.0, 1e-9])
+        if rc == 7:
+            break
+        served += rg[ro[1]:ro[2]].tolist()
+    assert served == [[20, 10], [0, 10], [30, 3], [10, 7], [17, 3]]
+
+
+def test_shuffle_can_leave_a_shard_in_its_place():
+    # A uniform shuffle of two shards keeps their order for about half of the seeds; a shuffle
+    # that always moves every element (a cyclic permutation) would swap them for every seed.
+    first = []
+    for seed in range(1, 65):
+        d = oracle.Dds(20, 10, 1, 1, seed)
+        rc, bsz, ro, rg, cnt = d.plan(None)
+        first.append(int(rg[0][0]))
+    assert 16 <= first.count(0) <= 48 and first.count(0) + first.count(10) == 64
 
 
 def test_doing_shard_is_exclusive_and_requeue_goes_to_queue_end():
